@@ -1,0 +1,302 @@
+"""Pins of the CPU oracle, step by step, against things other than itself:
+explicit matrices, closed forms, library routines, brute force, published known answers."""
+import itertools
+import math
+import os
+
+import numpy as np
+import pytest
+import scipy.linalg
+import torch
+
+import oracle as O
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def read_golden(name):
+    out = {}
+    with open(os.path.join(GOLD, name)) as f:
+        for line in f:
+            line = line.split("#")[0].strip()
+            if line:
+                k, v = line.split(None, 1)
+                out[k] = v.strip()
+    return out
+
+
+# ---------------------------------------------------------------- Hadamard (Sec. 2, Eq. 4)
+
+@pytest.mark.parametrize("G", [8, 16, 32, 64, 128])
+def test_butterfly_is_the_sylvester_matrix(G):
+    H = scipy.linalg.hadamard(G).astype(np.float64)          # library routine, natural order
+    c32 = np.float32(1.0 / math.sqrt(G))
+    rng = np.random.default_rng(G)
+    for _ in range(20):
+        x = rng.integers(-1000, 1000, G).astype(np.float32)
+        want = (np.float32(1) * (x.astype(np.float64) @ H).astype(np.float32)) * c32   # exact ints, one multiply
+        got = O.swap_hadamard(x, 0)                          # d = 0: the swap is the identity
+        assert np.array_equal(got, want)
+
+
+@pytest.mark.parametrize("G", [16, 64])
+def test_hadamard_orthogonality_and_involution(G):
+    # rows of the matrix the oracle applies, recovered from unit vectors; 1/sqrt(G) is a power of two here
+    M = np.stack([O.swap_hadamard(np.eye(G, dtype=np.float32)[i], 0) for i in range(G)]) * math.sqrt(G)
+    assert set(np.unique(M)) == {-1.0, 1.0}
+    assert np.array_equal(M @ M.T, G * np.eye(G))            # H H^T = G I
+    assert np.array_equal(M, M.T)                            # symmetric: the receiver reuses it
+    rng = np.random.default_rng(1)
+    x = rng.integers(-500, 500, G).astype(np.float32)
+    assert np.array_equal(O.swap_hadamard(O.swap_hadamard(x, 0), 0), x)
+
+
+@pytest.mark.parametrize("G", [32, 128])
+def test_hadamard_orthonormal_when_scale_is_irrational(G):
+    M = np.stack([O.swap_hadamard(np.eye(G, dtype=np.float32)[i], 0) for i in range(G)]).astype(np.float64)
+    assert np.allclose(M @ M.T, np.eye(G), atol=1e-6)
+    rng = np.random.default_rng(2)
+    x = rng.standard_normal(G).astype(np.float32)
+    y = O.swap_hadamard(x, 0)
+    assert abs(np.linalg.norm(y.astype(np.float64)) / np.linalg.norm(x.astype(np.float64)) - 1) < 1e-6
+
+
+def test_pivot_swap_is_a_transposition():
+    rng = np.random.default_rng(3)
+    G = 64
+    x = rng.integers(-99, 99, G).astype(np.float32)
+    for d in [0, 1, 17, 63]:
+        xs = x.copy()
+        xs[0], xs[d] = x[d], x[0]
+        assert np.array_equal(O.swap_hadamard(x, d), O.swap_hadamard(xs, 0))
+    # receiver: same butterfly, then the same swap, returns the tile (exact for small integers, G = 64)
+    d = 17
+    y = O.swap_hadamard(x, d)
+    back = O.swap_hadamard(y, 0)
+    back[0], back[d] = back[d], back[0]
+    assert np.array_equal(back, x)
+
+
+def test_one_hot_becomes_a_constant_tile():
+    # Sec. 3.3: after swap + H the former pivot is spread over all coordinates
+    G = 64
+    x = np.zeros(G, np.float32)
+    x[41] = 800.0
+    y = O.swap_hadamard(x, 41)
+    assert np.array_equal(y, np.full(G, 100.0, np.float32))
+
+
+# ---------------------------------------------------------------- outlier test (Eq. 3)
+
+def test_pivot_rule():
+    G = 64
+    base = np.full(G, 1.0, np.float32)
+    x = base.copy(); x[9] = 2.0
+    assert O.pivot(x) == (9, False)                       # r = 2/(1+1e-8) is not > 2
+    x[9] = 2.001
+    assert O.pivot(x) == (9, True)
+    x[9] = -2.001                                         # magnitudes decide
+    assert O.pivot(x) == (9, True)
+    x = base.copy(); x[5] = 3.0; x[50] = 3.0              # duplicated maximum: second largest equals it
+    assert O.pivot(x) == (5, False)
+    x = base.copy(); x[5] = -3.0; x[50] = 3.0             # first index wins the tie
+    assert O.pivot(x)[0] == 5
+    assert O.pivot(np.zeros(G, np.float32)) == (0, False)
+    one = np.zeros(G, np.float32); one[63] = 1e-3
+    assert O.pivot(one) == (63, True)
+
+
+def test_tau_extremes():
+    rng = np.random.default_rng(4)
+    for _ in range(50):
+        x = rng.standard_normal(32).astype(np.float32)
+        assert O.pivot(x, tau=0.0)[1] is True              # tau = 0: always transform
+        assert O.pivot(x, tau=float("inf"))[1] is False    # tau = inf: never
+        d, _ = O.pivot(x)
+        assert d == int(np.argmax(np.abs(x)))
+    assert O.pivot(np.zeros(32, np.float32), tau=0.0)[1] is False
+
+
+def test_pivot_flag_matches_ratio_definition():
+    rng = np.random.default_rng(5)
+    for _ in range(2000):
+        x = (rng.standard_normal(64) * np.exp(rng.standard_normal(64))).astype(np.float32)
+        a = np.sort(np.abs(x).astype(np.float64))[::-1]
+        r = a[0] / (a[1] + 1e-8)
+        if abs(r - 2.0) > 1e-5:                             # away from the rounding boundary
+            assert O.pivot(x)[1] == (r > 2.0)
+
+
+# ---------------------------------------------------------------- entropy (Eq. 1-2)
+
+def test_lg2_against_log2_all_mantissas():
+    m = (np.arange(2 ** 23, dtype=np.uint32) | np.uint32(0x3F800000)).view(np.float32)
+    err = O.lg2(m).astype(np.float64) - np.log2(m.astype(np.float64))
+    assert np.abs(err).max() < 3e-6
+    for e in [-27, -13, -1, 3]:
+        x = np.ldexp(m[::97], e).astype(np.float32)
+        err = O.lg2(x).astype(np.float64) - np.log2(x.astype(np.float64))
+        assert np.abs(err).max() < 3e-6 + 2.0 ** -24 * (abs(e) + 1)     # plus half an ulp of the result
+    k = np.arange(-30, 10)
+    assert np.array_equal(O.lg2(np.ldexp(np.float32(1), k)), k.astype(np.float32))   # exact at powers of two
+
+
+def test_treesum_order():
+    # exact for integers; the order is neighbours-first (distinguishes it from a running sum
+    # and from a stride-halving tree, which both give 2^24 here)
+    rng = np.random.default_rng(6)
+    x = rng.integers(-1000, 1000, 64).astype(np.float32)
+    assert O.treesum(x) == float(x.astype(np.int64).sum())
+    assert O.treesum(np.array([2 ** 24, 0, 1, 1], np.float32)) == 2 ** 24 + 2
+    assert O.treesum(np.array([1, 1, 2 ** 24, 0], np.float32)) == 2 ** 24 + 2
+
+
+@pytest.mark.parametrize("G", [8, 32, 64, 128])
+def test_entropy_closed_forms(G):
+    assert abs(O.score(np.ones(G)) - math.log2(G)) < 1e-4          # evenly spread: log2 G
+    assert abs(O.score(-7.5 * np.ones(G)) - math.log2(G)) < 1e-4   # magnitudes only
+    one = np.zeros(G); one[G // 3] = 123.0
+    assert abs(O.score(one)) < 1e-4                                # a single spike: 0
+    z = O.score(np.zeros(G))
+    assert z == 0.0 and not math.copysign(1, z) < 0                # +0, never -0
+    half = np.zeros(G); half[: G // 2] = 2.0
+    assert abs(O.score(half) - math.log2(G // 2)) < 1e-4
+    assert O.score(np.ones(G)) > O.score(half) > O.score(one)      # the sign the prose fixes
+
+
+def test_entropy_against_shannon_in_float64():
+    rng = np.random.default_rng(7)
+    for G in (32, 64, 128):
+        for _ in range(300):
+            x = (rng.standard_normal(G) * np.exp(2 * rng.standard_normal(G))).astype(np.float32)
+            a = np.abs(x.astype(np.float64))
+            p = a / (a.sum() + 1e-8)
+            H = -(p * np.log2(p + 1e-8)).sum()
+            assert abs(O.score(x) - H) < 2e-5
+            assert -1e-5 <= O.score(x) <= math.log2(G) + 1e-5
+
+
+# ---------------------------------------------------------------- allocation (Sec. 3.2)
+
+def test_allocation_brute_force():
+    rng = np.random.default_rng(8)
+    for trial in range(200):
+        n = int(rng.integers(1, 11))
+        k = int(rng.integers(0, n + 1))
+        s = rng.integers(0, 4, n).astype(np.float32)              # many ties
+        got = O.allocate(s, k)
+        assert got.sum() == k
+        best = None
+        for sub in itertools.combinations(range(n), k):           # all ways to hand out k high widths
+            key = (-sum(int(s[i]) for i in sub), sub)              # max total score, then lowest indices
+            if best is None or key < best:
+                best = key
+        want = np.zeros(n, np.uint8)
+        want[list(best[1])] = 1
+        assert np.array_equal(got, want)
+
+
+def test_allocation_with_float_scores_and_negatives():
+    s = np.array([0.5, -1e-7, 0.5, 3.0, 0.0, 0.5], np.float32)
+    assert O.allocate(s, 3).tolist() == [1, 0, 1, 1, 0, 0]
+    assert O.allocate(s, 5).tolist() == [1, 0, 1, 1, 1, 1]
+    assert O.allocate(s, 0).tolist() == [0] * 6
+    assert O.allocate(s, 6).tolist() == [1] * 6
+
+
+# ---------------------------------------------------------------- number formats
+
+def test_f16_against_numpy():
+    allh = np.arange(65536, dtype=np.uint16)
+    ref = allh.view(np.float16).astype(np.float32)
+    got = np.array([O.f16_to_f32(int(h)) for h in allh], np.float32)
+    assert np.array_equal(got.view(np.uint32), ref.view(np.uint32)) or np.array_equal(
+        got[~np.isnan(ref)], ref[~np.isnan(ref)])
+    rng = np.random.default_rng(9)
+    with np.errstate(invalid="ignore"):
+        ties = ((ref[:-1].astype(np.float64) + ref[1:].astype(np.float64)) / 2)[::5].astype(np.float32)
+    xs = np.concatenate([
+        (rng.standard_normal(20000) * np.exp(6 * rng.standard_normal(20000))).astype(np.float32),
+        np.ldexp(rng.standard_normal(20000), -20).astype(np.float32),        # half subnormals
+        ref[np.isfinite(ref)][::7],                                           # exact halves
+        ties,                                                                 # halfway cases
+    ])
+    xs = xs[np.isfinite(xs) & (np.abs(xs) <= 65504)]
+    with np.errstate(over="ignore"):
+        want = xs.astype(np.float16).view(np.uint16)
+    got = np.array([O.f32_to_f16(float(v)) for v in xs], np.uint16)
+    assert np.array_equal(got, want)
+
+
+def test_bf16_against_torch():
+    rng = np.random.default_rng(10)
+    xs = (rng.standard_normal(20000) * np.exp(8 * rng.standard_normal(20000))).astype(np.float32)
+    want = torch.from_numpy(xs).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    got = np.array([O.f32_to_bf16(float(v)) for v in xs], np.uint16)
+    assert np.array_equal(got, want)
+
+
+# ---------------------------------------------------------------- quantiser (Sec. 3.3)
+
+@pytest.mark.parametrize("bits", [2, 3, 4, 6, 8])
+def test_quantiser_is_textbook_minmax(bits):
+    rng = np.random.default_rng(11 + bits)
+    qmax = np.float32(2 ** bits - 1)
+    for _ in range(200):
+        v = (rng.standard_normal(64) * 3 + rng.standard_normal()).astype(np.float32)
+        sh, zh = O.tile_range(v, bits)
+        z = np.float32(np.float16(v.min()))                               # zero-point = min, in binary16
+        s = np.float32(np.float16((v.max() - z) / qmax))                  # scale = range / (2^b - 1)
+        assert zh == int(np.float16(v.min()).view(np.uint16))
+        assert sh == int(np.float16(s).view(np.uint16))
+        q = O.quantise(v, bits, sh, zh)
+        want = np.clip(np.rint((v - z) * (np.float32(1) / s)), 0, qmax).astype(np.uint32)
+        assert np.array_equal(q, want)
+        # error bound: half a step plus the binary16 rounding of z and s
+        xhat = z + q.astype(np.float32) * s
+        bound = s / 2 + abs(z - v.min()) + qmax * abs(float(s) - float((v.max() - z) / qmax)) + 1e-6
+        assert np.abs(xhat - v).max() <= bound
+
+
+def test_quantiser_degenerate_tiles():
+    v = np.full(64, 3.14159, np.float32)                       # flat: stored z may sit above max
+    sh, zh = O.tile_range(v, 4)
+    q = O.quantise(v, 4, sh, zh)
+    assert q.max() <= 15
+    s, z = O.f16_to_f32(sh), O.f16_to_f32(zh)
+    assert np.abs(z + q * s - v).max() <= 2 ** -11 * 3.2
+    v = np.zeros(64, np.float32); v[3] = -0.0
+    sh, zh = O.tile_range(v, 3)
+    assert (sh, zh) == (0, 0)                                   # -0 canonicalised
+    assert not O.quantise(v, 3, sh, zh).any()
+    big = np.linspace(-1e6, 1e6, 64).astype(np.float32)         # beyond binary16: saturates, stays in range
+    sh, zh = O.tile_range(big, 4)
+    assert zh == 0xFBFF and O.quantise(big, 4, sh, zh).max() <= 15
+
+
+# ---------------------------------------------------------------- stochastic rounding (optional mode)
+
+def test_philox_known_answers():
+    g = read_golden("philox4x32_10_kat.txt")
+    for i in range(3):
+        w = [int(t, 16) for t in g[f"kat{i}"].split()]
+        got = O.philox4x32_10(w[4:6], w[0:4])
+        assert [int(v) for v in got] == w[6:10]
+
+
+def test_stochastic_rounding_is_unbiased_and_bounded():
+    v = np.linspace(0.0, 15.0, 64).astype(np.float32) * np.float32(0.37) + np.float32(0.11)
+    sh, zh = O.tile_range(v, 4)
+    s, z = O.f16_to_f32(sh), O.f16_to_f32(zh)
+    acc = np.zeros(64)
+    n = 4000
+    for seed in range(n):
+        q = O.quantise(v, 4, sh, zh, rounding=1, seed=seed, first_elem=128)
+        assert q.max() <= 15
+        acc += q
+    y = (v - z) / s
+    assert np.abs(acc / n - np.clip(y, 0, 15)).max() < 0.04     # E[q] = y
+    a = O.quantise(v, 4, sh, zh, rounding=1, seed=5, first_elem=128)
+    b = O.quantise(v, 4, sh, zh, rounding=1, seed=5, first_elem=128)
+    assert np.array_equal(a, b)                                  # counter-based: reproducible
+    assert np.abs(a.astype(np.float64) - y).max() < 1.0 + 1e-3
