@@ -1,0 +1,142 @@
+/*
+ * tahq.h -- C ABI of the B200 (sm_100a) TAH-Quant boundary codec.
+ *
+ * The library compresses the activation (or activation-gradient) tensor that
+ * crosses a pipeline-stage boundary and restores it on the other side
+ * (TAH-Quant, Sec. 3.1-3.4; Algorithm 1 lines 4-5).  All work runs in CUDA
+ * kernels on the caller's stream; there is no CPU fallback.
+ *
+ * Conventions for every entry point
+ *   - Pointers named d_* are DEVICE pointers, 16-byte aligned, owned by the
+ *     caller.  The library never allocates, frees or synchronises, and never
+ *     touches a stream other than the one passed in.
+ *   - Calls are asynchronous and stream-ordered.  Host-detectable errors are
+ *     returned before anything is enqueued.
+ *   - d_ws is scratch memory of at least tahq_workspace_bound() bytes.  Its
+ *     first 4 bytes are a device status word (0 = ok, see TAHQ_DEV_*) that the
+ *     caller may read after synchronising the stream.  Two calls that overlap
+ *     on the GPU must not share a workspace.
+ *   - Inputs must be finite.  Non-finite inputs give unspecified values but
+ *     never touch memory outside the buffers.
+ *   - Same inputs, same bytes: every byte of [0, tahq_packed_bound()) is
+ *     written, padding included.
+ */
+#ifndef TAHQ_H
+#define TAHQ_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* Opaque stand-in for cudaStream_t so that this header needs no CUDA include. */
+typedef struct CUstream_st *tahq_stream;
+
+typedef enum {
+  TAHQ_OK = 0,
+  TAHQ_ERR_INVALID_ARG = 1,      /* null pointer, bad struct_size, bad shape/tile/budget        */
+  TAHQ_ERR_UNSUPPORTED = 2,      /* valid in the format but not built (e.g. tile < 32)          */
+  TAHQ_ERR_BUFFER_TOO_SMALL = 3, /* packed_cap / packed_bytes / ws_cap below the bound          */
+  TAHQ_ERR_MISALIGNED = 4,       /* a device pointer is not 16-byte aligned                     */
+  TAHQ_ERR_CUDA = 5              /* a CUDA runtime call (launch, memset) failed                 */
+} tahq_status;
+
+typedef enum { TAHQ_F32 = 0, TAHQ_BF16 = 1 } tahq_dtype;
+
+/* Bits of the device status word at d_ws[0..4). */
+enum {
+  TAHQ_DEV_OK = 0,
+  TAHQ_DEV_BAD_HEADER = 1,       /* decode: the buffer's header does not match the parameters   */
+  TAHQ_DEV_BAD_BITMAP = 2,       /* decode: bit map population does not match the payload size  */
+  TAHQ_DEV_TIMEOUT = 4           /* a bounded device-side wait ran out                          */
+};
+
+/*
+ * One boundary tensor.  Names follow the paper: a tile is a quantisation group
+ * of G contiguous channels of one token (Sec. 3.1); allocation tiles equal
+ * quantisation tiles (A = G, the default of Sec. 3.2); a ranking group is one
+ * sample of S = group_tokens consecutive tokens (Sec. 3.2, top-p% selection).
+ */
+typedef struct {
+  uint32_t struct_size;      /* = sizeof(tahq_params)                                            */
+  uint32_t dtype;            /* tahq_dtype of the dense row-major [tokens x hidden] tensor       */
+  uint64_t tokens;           /* T = B*S                                                          */
+  uint32_t hidden;           /* C, a multiple of tile                                            */
+  uint32_t group_tokens;     /* S; 0 = the whole tensor is one ranking group; must divide T      */
+  uint32_t tile;             /* G in {32, 64, 128}                                               */
+  uint32_t budget_millibits; /* payload bits per element x 1000, in [2000, 8000].  lo = b/1000
+                                bits for every tile, and the floor(n_g*(b%1000)/1000) highest-
+                                entropy tiles of each ranking group get lo+1.  3800 is the
+                                paper's 80% INT4 + 20% INT3.                                     */
+  float tau;                 /* outlier threshold of Eq. 3 (paper: 2.0; 0 = always transform,
+                                +inf = never)                                                    */
+  float eps_l1;              /* epsilon  of Eq. 1 (1e-8f)                                        */
+  float eps_log;             /* varsigma of Eq. 2 (1e-8f)                                        */
+  float eps_ratio;           /* varrho   of Eq. 3 (1e-8f)                                        */
+  uint32_t rounding;         /* 0 = round-half-even; 1 = stochastic (Philox4x32-10 keyed by seed,
+                                counter = element index / 4)                                     */
+  uint64_t seed;             /* used only when rounding == 1                                     */
+} tahq_params;
+
+/* Byte offsets of the sections of the packed buffer (all multiples of 128). */
+typedef struct {
+  uint64_t n_tiles, n_groups, tiles_per_group, k_hi;
+  uint32_t lo_bits, hi_bits;
+  uint64_t off_bitmap, off_scale_zero, off_pivot, off_payload;
+  uint64_t payload_bytes, total_bytes;
+} tahq_layout;
+
+/*
+ * Exact size in bytes of the packed buffer (Sec. 3.4: a fixed-shape uint8
+ * stream; the size depends on the parameters only, never on the data).
+ * Returns 0 when the parameters are invalid or unsupported.  Host-only.
+ */
+size_t tahq_packed_bound(const tahq_params *p);
+
+/* Section offsets of the packed buffer; TAHQ_OK or an error.  Host-only. */
+tahq_status tahq_packed_layout(const tahq_params *p, tahq_layout *out);
+
+/*
+ * Bytes of scratch that tahq_encode / tahq_decode need for these parameters
+ * (tile scores, selection histograms and candidates, offset prefixes, status
+ * word).  Returns 0 when the parameters are invalid.  Host-only.
+ */
+size_t tahq_workspace_bound(const tahq_params *p);
+
+/*
+ * Encode (Sec. 3.1-3.4): d_in [tokens x hidden] (dtype) -> d_packed.
+ *   Per tile: entropy score on the raw tile (Eq. 1-2); per ranking group the
+ *   top-p% scores get the higher width (Sec. 3.2); outlier test (Eq. 3), pivot
+ *   swap + Hadamard on flagged tiles (Eq. 4); min-max asymmetric quantisation
+ *   with binary16 scale and zero-point (Sec. 3.3); variable-width little-endian
+ *   bit packing plus bit map, scale/zero and pivot sections (Sec. 3.4).
+ * d_in is read only; d_packed[0, packed_bound) is fully overwritten.
+ * Errors: INVALID_ARG, UNSUPPORTED, BUFFER_TOO_SMALL (packed_cap or ws_cap),
+ * MISALIGNED, CUDA.  Nothing is enqueued when an error is returned.
+ */
+tahq_status tahq_encode(const tahq_params *p, const void *d_in, void *d_packed, size_t packed_cap,
+                        void *d_ws, size_t ws_cap, tahq_stream stream);
+
+/*
+ * Decode (Sec. 3.3, Algorithm 1 line 5): d_packed -> d_out [tokens x hidden]
+ * (dtype): bit map -> widths and offsets, unpack, z + q*s, inverse Hadamard
+ * and un-swap on flagged tiles, store (round-to-nearest-even for bf16).
+ * The header inside d_packed must describe the same parameters; a mismatch is
+ * reported through the device status word and the output is left untouched.
+ * Errors as for tahq_encode (packed_bytes must be >= tahq_packed_bound()).
+ */
+tahq_status tahq_decode(const tahq_params *p, const void *d_packed, size_t packed_bytes, void *d_out,
+                        void *d_ws, size_t ws_cap, tahq_stream stream);
+
+/* Static string for a status code. */
+const char *tahq_status_string(tahq_status s);
+
+/* Number of kernels the last tahq_encode / tahq_decode call of this thread enqueued. */
+int tahq_last_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TAHQ_H */

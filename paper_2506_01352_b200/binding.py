@@ -1,0 +1,187 @@
+"""ctypes binding of the C ABI in include/tahq.h (argument marshalling only).
+
+Every step of encode and decode runs in the CUDA kernels of ``libtahq.so``; PyTorch is used here
+for device memory and streams.  There is no CPU fallback: importing this module without the built
+library raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+
+import torch
+
+from . import build as _build
+
+F32, BF16 = 0, 1
+OK = 0
+DEV_OK, DEV_BAD_HEADER, DEV_BAD_BITMAP, DEV_TIMEOUT = 0, 1, 2, 4
+
+
+class _Params(C.Structure):
+    _fields_ = [
+        ("struct_size", C.c_uint32), ("dtype", C.c_uint32), ("tokens", C.c_uint64), ("hidden", C.c_uint32),
+        ("group_tokens", C.c_uint32), ("tile", C.c_uint32), ("budget_millibits", C.c_uint32),
+        ("tau", C.c_float), ("eps_l1", C.c_float), ("eps_log", C.c_float), ("eps_ratio", C.c_float),
+        ("rounding", C.c_uint32), ("seed", C.c_uint64),
+    ]
+
+
+class _Layout(C.Structure):
+    _fields_ = [
+        ("n_tiles", C.c_uint64), ("n_groups", C.c_uint64), ("tiles_per_group", C.c_uint64), ("k_hi", C.c_uint64),
+        ("lo_bits", C.c_uint32), ("hi_bits", C.c_uint32), ("off_bitmap", C.c_uint64),
+        ("off_scale_zero", C.c_uint64), ("off_pivot", C.c_uint64), ("off_payload", C.c_uint64),
+        ("payload_bytes", C.c_uint64), ("total_bytes", C.c_uint64),
+    ]
+
+
+@dataclass
+class Params:
+    """tahq_params: one boundary tensor [tokens x hidden]; G = tile, S = group_tokens (paper notation)."""
+
+    tokens: int
+    hidden: int
+    dtype: int = F32
+    group_tokens: int = 0
+    tile: int = 64
+    budget_millibits: int = 3800
+    tau: float = 2.0
+    eps_l1: float = 1e-8
+    eps_log: float = 1e-8
+    eps_ratio: float = 1e-8
+    rounding: int = 0
+    seed: int = 0
+
+    def c(self) -> _Params:
+        return _Params(C.sizeof(_Params), self.dtype, self.tokens, self.hidden, self.group_tokens, self.tile,
+                       self.budget_millibits, self.tau, self.eps_l1, self.eps_log, self.eps_ratio,
+                       self.rounding, self.seed)
+
+
+class TahqError(RuntimeError):
+    def __init__(self, code: int):
+        self.code = code
+        super().__init__(f"tahq: {status_string(code)} ({code})")
+
+
+EXPORTS = ["tahq_packed_bound", "tahq_packed_layout", "tahq_workspace_bound", "tahq_encode", "tahq_decode",
+           "tahq_status_string", "tahq_last_launch_count"]
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """Load libtahq.so (built in-tree).  Raises if it is missing: there is no other implementation."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_build.LIB):
+            raise ImportError(f"{_build.LIB} is not built; run `python -c 'import __graft_entry__ as g; g.build()'`")
+        L = C.CDLL(_build.LIB)
+        pp = C.POINTER(_Params)
+        L.tahq_packed_bound.argtypes = [pp]
+        L.tahq_packed_bound.restype = C.c_size_t
+        L.tahq_packed_layout.argtypes = [pp, C.POINTER(_Layout)]
+        L.tahq_packed_layout.restype = C.c_int
+        L.tahq_workspace_bound.argtypes = [pp]
+        L.tahq_workspace_bound.restype = C.c_size_t
+        L.tahq_encode.argtypes = [pp, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p, C.c_size_t, C.c_void_p]
+        L.tahq_encode.restype = C.c_int
+        L.tahq_decode.argtypes = [pp, C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+        L.tahq_decode.restype = C.c_int
+        L.tahq_status_string.argtypes = [C.c_int]
+        L.tahq_status_string.restype = C.c_char_p
+        L.tahq_last_launch_count.argtypes = []
+        L.tahq_last_launch_count.restype = C.c_int
+        _lib = L
+    return _lib
+
+
+def status_string(code: int) -> str:
+    return lib().tahq_status_string(int(code)).decode()
+
+
+def packed_bound(p: Params) -> int:
+    pc = p.c()
+    return int(lib().tahq_packed_bound(C.byref(pc)))
+
+
+def workspace_bound(p: Params) -> int:
+    pc = p.c()
+    return int(lib().tahq_workspace_bound(C.byref(pc)))
+
+
+def packed_layout(p: Params) -> dict:
+    pc, out = p.c(), _Layout()
+    rc = lib().tahq_packed_layout(C.byref(pc), C.byref(out))
+    if rc != OK:
+        raise TahqError(rc)
+    return {k: int(getattr(out, k)) for k, _ in _Layout._fields_}
+
+
+def last_launch_count() -> int:
+    return int(lib().tahq_last_launch_count())
+
+
+def _stream_handle(stream) -> int:
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return int(s.cuda_stream)
+
+
+def tahq_encode(p: Params, d_in: int, d_packed: int, packed_cap: int, d_ws: int, ws_cap: int, stream: int) -> int:
+    """Raw call: device addresses as integers, returns the tahq_status."""
+    pc = p.c()
+    return int(lib().tahq_encode(C.byref(pc), d_in, d_packed, packed_cap, d_ws, ws_cap, stream))
+
+
+def tahq_decode(p: Params, d_packed: int, packed_bytes: int, d_out: int, d_ws: int, ws_cap: int, stream: int) -> int:
+    pc = p.c()
+    return int(lib().tahq_decode(C.byref(pc), d_packed, packed_bytes, d_out, d_ws, ws_cap, stream))
+
+
+def params_for(x: torch.Tensor, **kw) -> Params:
+    if x.dim() != 2:
+        raise ValueError("expected a [tokens x hidden] tensor")
+    dt = {torch.float32: F32, torch.bfloat16: BF16}[x.dtype]
+    return Params(tokens=x.shape[0], hidden=x.shape[1], dtype=dt, **kw)
+
+
+def alloc_packed(p: Params, device="cuda") -> torch.Tensor:
+    return torch.empty(packed_bound(p), dtype=torch.uint8, device=device)
+
+
+def alloc_workspace(p: Params, device="cuda") -> torch.Tensor:
+    return torch.empty(workspace_bound(p), dtype=torch.uint8, device=device)
+
+
+def encode(p: Params, x: torch.Tensor, packed: torch.Tensor | None = None, ws: torch.Tensor | None = None,
+           stream=None) -> torch.Tensor:
+    """Encode a contiguous CUDA tensor; returns the packed uint8 buffer (asynchronous on the stream)."""
+    if not (x.is_cuda and x.is_contiguous()):
+        raise ValueError("x must be a contiguous CUDA tensor")
+    packed = alloc_packed(p, x.device) if packed is None else packed
+    ws = alloc_workspace(p, x.device) if ws is None else ws
+    rc = tahq_encode(p, x.data_ptr(), packed.data_ptr(), packed.numel(), ws.data_ptr(), ws.numel(),
+                     _stream_handle(stream))
+    if rc != OK:
+        raise TahqError(rc)
+    return packed
+
+
+def decode(p: Params, packed: torch.Tensor, out: torch.Tensor | None = None, ws: torch.Tensor | None = None,
+           stream=None) -> torch.Tensor:
+    if out is None:
+        out = torch.empty(p.tokens, p.hidden, dtype=torch.float32 if p.dtype == F32 else torch.bfloat16,
+                          device=packed.device)
+    ws = alloc_workspace(p, packed.device) if ws is None else ws
+    rc = tahq_decode(p, packed.data_ptr(), packed.numel(), out.data_ptr(), ws.data_ptr(), ws.numel(),
+                     _stream_handle(stream))
+    if rc != OK:
+        raise TahqError(rc)
+    return out
+
+
+def device_status(ws: torch.Tensor) -> int:
+    """Device status word of the last call that used this workspace (synchronises)."""
+    return int(ws[:4].view(torch.int32).item())

@@ -1,0 +1,301 @@
+// Host side of the C ABI declared in include/tahq.h: parameter validation, layout of the packed
+// buffer and of the workspace, kernel selection and launches on the caller's stream.
+#include "../../include/tahq.h"
+
+#include <atomic>
+#include <cstring>
+
+#include "tahq_kernels.cuh"
+
+namespace tahq {
+
+static thread_local int g_launches = 0;
+
+struct Plan {
+  tahq_layout L;
+  uint32_t f;             // budget % 1000
+  bool mixed;             // two widths in use (k_hi > 0)
+  bool direct;            // small ranking groups: select straight from the scores
+  uint32_t cpg, cand_cap;
+  uint64_t n128;
+  // workspace offsets
+  uint64_t ws_ncand, ws_hist, ws_zero_end, ws_scores, ws_binsel, ws_theta, ws_cand, ws_cnt, ws_total;
+};
+
+static uint64_t up(uint64_t x, uint64_t a) { return (x + a - 1) / a * a; }
+
+static tahq_status make_plan(const tahq_params *p, Plan *pl) {
+  if (!p || p->struct_size != sizeof(tahq_params)) return TAHQ_ERR_INVALID_ARG;
+  const uint32_t G = p->tile;
+  if (G < 8 || G > 128 || (G & (G - 1))) return TAHQ_ERR_INVALID_ARG;
+  if (p->dtype > 1 || p->rounding > 1) return TAHQ_ERR_INVALID_ARG;
+  if (p->tokens == 0 || p->hidden == 0 || p->hidden % G) return TAHQ_ERR_INVALID_ARG;
+  const uint64_t S = p->group_tokens ? p->group_tokens : p->tokens;
+  if (p->tokens % S) return TAHQ_ERR_INVALID_ARG;
+  const uint32_t beta = p->budget_millibits;
+  if (beta < 2000 || beta > 8000) return TAHQ_ERR_INVALID_ARG;
+  if (!(p->tau >= 0.0f) || !(p->eps_l1 >= 0.0f) || !(p->eps_log >= 0.0f) || !(p->eps_ratio >= 0.0f))
+    return TAHQ_ERR_INVALID_ARG;
+  const uint64_t M = p->hidden / G;
+  if (p->tokens > (1ull << 40) / M) return TAHQ_ERR_INVALID_ARG;
+  tahq_layout &L = pl->L;
+  L.n_tiles = p->tokens * M;
+  L.tiles_per_group = S * M;
+  L.n_groups = p->tokens / S;
+  if (L.tiles_per_group >= (1ull << 32) || L.n_tiles >= (1ull << 36)) return TAHQ_ERR_INVALID_ARG;
+  pl->f = beta % 1000;
+  L.lo_bits = beta / 1000;
+  L.hi_bits = pl->f ? L.lo_bits + 1 : L.lo_bits;
+  L.k_hi = L.tiles_per_group * (uint64_t)pl->f / 1000u;
+  L.payload_bytes = L.n_groups * (uint64_t)(G / 8) * (L.tiles_per_group * L.lo_bits + L.k_hi);
+  L.off_bitmap = 128;
+  L.off_scale_zero = up(L.off_bitmap + (L.n_tiles + 7) / 8, 128);
+  L.off_pivot = up(L.off_scale_zero + 4 * L.n_tiles, 128);
+  L.off_payload = up(L.off_pivot + L.n_tiles, 128);
+  L.total_bytes = up(L.off_payload + L.payload_bytes, 128);
+  if (G < 32) return TAHQ_ERR_UNSUPPORTED;
+  if (p->rounding != 0) return TAHQ_ERR_UNSUPPORTED;
+
+  pl->mixed = L.k_hi > 0;
+  pl->direct = L.tiles_per_group <= 16384;
+  pl->cpg = 1;
+  pl->cand_cap = 0;
+  if (pl->mixed && !pl->direct) {
+    uint64_t cpg = (L.tiles_per_group + 8191) / 8192;
+    pl->cpg = (uint32_t)(cpg > 128 ? 128 : cpg);
+    pl->cand_cap = (uint32_t)(L.tiles_per_group < 32768 ? L.tiles_per_group : 32768);
+  }
+  pl->n128 = (L.n_tiles + 127) / 128;
+  uint64_t o = 256;                                         // status word and friends
+  pl->ws_ncand = o;  o = up(o + 4 * L.n_groups, 256);
+  pl->ws_hist = o;   o += (pl->mixed && !pl->direct) ? 4ull * kBins * L.n_groups : 0;
+  pl->ws_zero_end = o;                                      // [0, ws_zero_end) is cleared per call
+  pl->ws_scores = o; o = up(o + (pl->mixed ? 4 * L.n_tiles : 0), 256);
+  pl->ws_binsel = o; o = up(o + 8 * L.n_groups, 256);
+  pl->ws_theta = o;  o = up(o + 8 * L.n_groups, 256);
+  pl->ws_cand = o;   o = up(o + 8ull * pl->cand_cap * L.n_groups, 256);
+  pl->ws_cnt = o;    o = up(o + 4 * (pl->n128 + 2), 256);
+  pl->ws_total = o;
+  return TAHQ_OK;
+}
+
+static void fill_header(const tahq_params *p, const Plan &pl, uint32_t *h) {
+  std::memset(h, 0, 128);
+  auto f2u = [](float f) { uint32_t u; std::memcpy(&u, &f, 4); return u; };
+  auto put64 = [&](int w, uint64_t v) { h[w] = (uint32_t)v; h[w + 1] = (uint32_t)(v >> 32); };
+  h[0] = 0x51484154u;  // "TAHQ"
+  h[1] = 1;
+  h[2] = p->dtype;
+  h[3] = p->rounding;
+  put64(4, p->tokens);
+  h[6] = p->hidden;
+  h[7] = p->tile;
+  h[8] = (uint32_t)(pl.L.tiles_per_group / (p->hidden / p->tile));
+  h[9] = p->budget_millibits;
+  h[10] = f2u(p->tau);
+  h[11] = f2u(p->eps_l1);
+  h[12] = f2u(p->eps_log);
+  h[13] = f2u(p->eps_ratio);
+  put64(14, p->seed);
+  put64(16, pl.L.n_tiles);
+  put64(18, pl.L.payload_bytes);
+  put64(20, pl.L.total_bytes);
+}
+
+static void fill_args(const tahq_params *p, const Plan &pl, uint8_t *ws, Args *a) {
+  std::memset(a, 0, sizeof(*a));
+  a->n_tiles = pl.L.n_tiles;
+  a->tiles_per_group = pl.L.tiles_per_group;
+  a->k_hi = pl.L.k_hi;
+  a->n_groups = pl.L.n_groups;
+  a->lo = pl.L.lo_bits;
+  a->mixed = pl.mixed;
+  a->off_bitmap = pl.L.off_bitmap;
+  a->off_sz = pl.L.off_scale_zero;
+  a->off_pivot = pl.L.off_pivot;
+  a->off_payload = pl.L.off_payload;
+  a->payload_bytes = pl.L.payload_bytes;
+  a->total_bytes = pl.L.total_bytes;
+  a->tau = p->tau;
+  a->eps_l1 = p->eps_l1;
+  a->eps_log = p->eps_log;
+  a->eps_ratio = p->eps_ratio;
+  a->status = reinterpret_cast<uint32_t *>(ws);
+  a->ncand = reinterpret_cast<uint32_t *>(ws + pl.ws_ncand);
+  a->hist = reinterpret_cast<uint32_t *>(ws + pl.ws_hist);
+  a->scores = reinterpret_cast<float *>(ws + pl.ws_scores);
+  a->binsel = reinterpret_cast<uint2 *>(ws + pl.ws_binsel);
+  a->theta = reinterpret_cast<unsigned long long *>(ws + pl.ws_theta);
+  a->cand = reinterpret_cast<unsigned long long *>(ws + pl.ws_cand);
+  a->cnt128 = reinterpret_cast<uint32_t *>(ws + pl.ws_cnt);
+  a->cand_cap = pl.cand_cap;
+  a->cpg = pl.cpg;
+  a->direct = pl.direct;
+  fill_header(p, pl, a->header);
+}
+
+// ---- launch helpers ----------------------------------------------------------------------
+
+struct DevInfo { int dev, sms; };
+static bool dev_info(DevInfo *d) {
+  if (cudaGetDevice(&d->dev) != cudaSuccess) return false;
+  return cudaDeviceGetAttribute(&d->sms, cudaDevAttrMultiProcessorCount, d->dev) == cudaSuccess;
+}
+
+// Opt a kernel into its dynamic shared memory once per device and return resident CTAs per SM.
+template <class K>
+static int prepare(K kernel, int smem, const DevInfo &d, std::atomic<int> *cache) {
+  int v = cache[d.dev & 63].load(std::memory_order_acquire);
+  if (v > 0) return v;
+  if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return 0;
+  int occ = 0;
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kernel, kThreads, smem) != cudaSuccess || occ < 1)
+    return 0;
+  cache[d.dev & 63].store(occ, std::memory_order_release);
+  return occ;
+}
+
+template <class C> struct Stages {
+  static constexpr int STATS = (C::ROWB == 256) ? 2 : (C::ROWB == 128 ? 3 : 4);
+  static constexpr int QUANT = (C::ROWB == 256) ? 3 : (C::ROWB == 128 ? 3 : 4);
+};
+
+template <class C>
+static tahq_status encode_t(const Plan &pl, const Args &a, cudaStream_t st) {
+  DevInfo d;
+  if (!dev_info(&d)) return TAHQ_ERR_CUDA;
+  const uint64_t n_chunks = (a.n_tiles + C::TPC - 1) / C::TPC;
+  static std::atomic<int> occ_stats[64], occ_quant[64];
+  if (pl.mixed) {
+    constexpr int NS = Stages<C>::STATS;
+    const int smem = NS * C::STAGE_BYTES;
+    const int occ = prepare(stats_kernel<C, NS>, smem, d, occ_stats);
+    if (!occ) return TAHQ_ERR_CUDA;
+    const uint64_t cap = (uint64_t)d.sms * occ;
+    stats_kernel<C, NS><<<(unsigned)(n_chunks < cap ? n_chunks : cap), kThreads, smem, st>>>(a);
+    ++g_launches;
+    if (!pl.direct) {
+      hist_kernel<<<(unsigned)(a.n_groups * a.cpg), kThreads, 0, st>>>(a);
+      gather_kernel<<<(unsigned)(a.n_groups * a.cpg), kThreads, 0, st>>>(a);
+      g_launches += 2;
+    }
+    resolve_kernel<<<(unsigned)a.n_groups, kResolveThreads, 0, st>>>(a);
+    bitmap_kernel<<<(unsigned)((a.n_tiles + kThreads - 1) / kThreads), kThreads, 0, st>>>(a);
+    scan_kernel<<<1, kScanThreads, 0, st>>>(a.cnt128, pl.n128, ~0ull, a.status);
+    g_launches += 3;
+  }
+  constexpr int NQ = Stages<C>::QUANT;
+  const int smem = NQ * C::STAGE_BYTES + C::MAX_PAY;
+  const int occ = prepare(quant_pack_kernel<C, NQ>, smem, d, occ_quant);
+  if (!occ) return TAHQ_ERR_CUDA;
+  const uint64_t cap = (uint64_t)d.sms * occ;
+  quant_pack_kernel<C, NQ><<<(unsigned)(n_chunks < cap ? n_chunks : cap), kThreads, smem, st>>>(a);
+  ++g_launches;
+  return cudaGetLastError() == cudaSuccess ? TAHQ_OK : TAHQ_ERR_CUDA;
+}
+
+template <class C>
+static tahq_status decode_t(const Plan &pl, const Args &a, cudaStream_t st) {
+  DevInfo d;
+  if (!dev_info(&d)) return TAHQ_ERR_CUDA;
+  const uint64_t n_chunks = (a.n_tiles + C::TPC - 1) / C::TPC;
+  static std::atomic<int> occ_dec[64];
+  count_kernel<<<(unsigned)((pl.n128 + kThreads - 1) / kThreads), kThreads, 0, st>>>(a);
+  scan_kernel<<<1, kScanThreads, 0, st>>>(a.cnt128, pl.n128, pl.mixed ? a.n_groups * a.k_hi : ~0ull, a.status);
+  const int smem = C::STAGE_BYTES;
+  const int occ = prepare(decode_kernel<C>, smem, d, occ_dec);
+  if (!occ) return TAHQ_ERR_CUDA;
+  const uint64_t cap = (uint64_t)d.sms * occ * 8;
+  decode_kernel<C><<<(unsigned)(n_chunks < cap ? n_chunks : cap), kThreads, smem, st>>>(a);
+  g_launches += 3;
+  return cudaGetLastError() == cudaSuccess ? TAHQ_OK : TAHQ_ERR_CUDA;
+}
+
+static bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+}  // namespace tahq
+
+using namespace tahq;
+
+extern "C" {
+
+size_t tahq_packed_bound(const tahq_params *p) {
+  Plan pl;
+  return make_plan(p, &pl) == TAHQ_OK ? (size_t)pl.L.total_bytes : 0;
+}
+
+tahq_status tahq_packed_layout(const tahq_params *p, tahq_layout *out) {
+  Plan pl;
+  const tahq_status s = make_plan(p, &pl);
+  if (s != TAHQ_OK) return s;
+  if (!out) return TAHQ_ERR_INVALID_ARG;
+  *out = pl.L;
+  return TAHQ_OK;
+}
+
+size_t tahq_workspace_bound(const tahq_params *p) {
+  Plan pl;
+  return make_plan(p, &pl) == TAHQ_OK ? (size_t)pl.ws_total : 0;
+}
+
+tahq_status tahq_encode(const tahq_params *p, const void *d_in, void *d_packed, size_t packed_cap, void *d_ws,
+                        size_t ws_cap, tahq_stream stream) {
+  g_launches = 0;
+  Plan pl;
+  const tahq_status s = make_plan(p, &pl);
+  if (s != TAHQ_OK) return s;
+  if (!d_in || !d_packed || !d_ws) return TAHQ_ERR_INVALID_ARG;
+  if (packed_cap < pl.L.total_bytes || ws_cap < pl.ws_total) return TAHQ_ERR_BUFFER_TOO_SMALL;
+  if (!aligned16(d_in) || !aligned16(d_packed) || !aligned16(d_ws)) return TAHQ_ERR_MISALIGNED;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  Args a;
+  fill_args(p, pl, static_cast<uint8_t *>(d_ws), &a);
+  a.in = static_cast<const uint8_t *>(d_in);
+  a.packed = static_cast<uint8_t *>(d_packed);
+  if (cudaMemsetAsync(d_ws, 0, pl.ws_zero_end, st) != cudaSuccess) return TAHQ_ERR_CUDA;
+  const bool bf = p->dtype == TAHQ_BF16;
+  switch (p->tile) {
+    case 32: return bf ? encode_t<Cfg<32, true>>(pl, a, st) : encode_t<Cfg<32, false>>(pl, a, st);
+    case 64: return bf ? encode_t<Cfg<64, true>>(pl, a, st) : encode_t<Cfg<64, false>>(pl, a, st);
+    default: return bf ? encode_t<Cfg<128, true>>(pl, a, st) : encode_t<Cfg<128, false>>(pl, a, st);
+  }
+}
+
+tahq_status tahq_decode(const tahq_params *p, const void *d_packed, size_t packed_bytes, void *d_out, void *d_ws,
+                        size_t ws_cap, tahq_stream stream) {
+  g_launches = 0;
+  Plan pl;
+  const tahq_status s = make_plan(p, &pl);
+  if (s != TAHQ_OK) return s;
+  if (!d_out || !d_packed || !d_ws) return TAHQ_ERR_INVALID_ARG;
+  if (packed_bytes < pl.L.total_bytes || ws_cap < pl.ws_total) return TAHQ_ERR_BUFFER_TOO_SMALL;
+  if (!aligned16(d_out) || !aligned16(d_packed) || !aligned16(d_ws)) return TAHQ_ERR_MISALIGNED;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  Args a;
+  fill_args(p, pl, static_cast<uint8_t *>(d_ws), &a);
+  a.packed = const_cast<uint8_t *>(static_cast<const uint8_t *>(d_packed));
+  a.out = static_cast<uint8_t *>(d_out);
+  if (cudaMemsetAsync(d_ws, 0, 256, st) != cudaSuccess) return TAHQ_ERR_CUDA;
+  const bool bf = p->dtype == TAHQ_BF16;
+  switch (p->tile) {
+    case 32: return bf ? decode_t<Cfg<32, true>>(pl, a, st) : decode_t<Cfg<32, false>>(pl, a, st);
+    case 64: return bf ? decode_t<Cfg<64, true>>(pl, a, st) : decode_t<Cfg<64, false>>(pl, a, st);
+    default: return bf ? decode_t<Cfg<128, true>>(pl, a, st) : decode_t<Cfg<128, false>>(pl, a, st);
+  }
+}
+
+const char *tahq_status_string(tahq_status s) {
+  switch (s) {
+    case TAHQ_OK: return "ok";
+    case TAHQ_ERR_INVALID_ARG: return "invalid argument";
+    case TAHQ_ERR_UNSUPPORTED: return "unsupported configuration";
+    case TAHQ_ERR_BUFFER_TOO_SMALL: return "buffer too small";
+    case TAHQ_ERR_MISALIGNED: return "pointer not 16-byte aligned";
+    case TAHQ_ERR_CUDA: return "CUDA runtime error";
+  }
+  return "unknown status";
+}
+
+int tahq_last_launch_count(void) { return g_launches; }
+
+}  // extern "C"

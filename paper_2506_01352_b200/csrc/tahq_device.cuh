@@ -1,0 +1,248 @@
+// Device-side building blocks of the TAH-Quant boundary codec for sm_100a.
+//
+// Work decomposition: ONE THREAD OWNS ONE TILE (quantisation group, Sec. 3.1) -- or half of a
+// 128-wide tile -- and keeps its elements in registers, so that the Hadamard butterfly (Eq. 4),
+// the reductions of Eq. 1-3 and the bit packing need no cross-lane traffic.  Tiles reach the
+// thread through shared memory: a CTA copies 256 thread-rows with 16-byte cp.async into an
+// XOR-swizzled stage from which every thread reads its own row with conflict-free 128-bit loads.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace tahq {
+
+constexpr int kThreads = 256;          // threads per CTA of the tile kernels
+constexpr int kBins = 4096;            // first-level histogram of the top-p% selection
+constexpr float kBinScale = 512.0f;    // bins per unit of score (scores lie in [0, log2 128])
+constexpr unsigned kFull = 0xffffffffu;
+
+// ------------------------------------------------------------------------------------------
+// Geometry of one (tile width, dtype) instantiation
+// ------------------------------------------------------------------------------------------
+template <int G_, bool BF16_>
+struct Cfg {
+  static constexpr int G = G_;
+  static constexpr bool BF16 = BF16_;
+  static constexpr int LPT = (G == 128) ? 2 : 1;   // lanes (threads) per tile
+  static constexpr int EPT = G / LPT;              // elements per thread: 32 or 64
+  static constexpr int ESZ = BF16 ? 2 : 4;
+  static constexpr int ROWB = EPT * ESZ;           // bytes of one thread-row: 64 / 128 / 256
+  static constexpr int CPR = ROWB / 16;            // 16-byte chunks per row: 4 / 8 / 16
+  static constexpr int TPC = kThreads / LPT;       // tiles per CTA chunk
+  static constexpr int STAGE_BYTES = kThreads * ROWB;
+  static constexpr int NOCT = EPT / 8;             // groups of 8 elements per thread
+  static constexpr int MAX_PAY = kThreads * EPT;   // payload bytes of one chunk at 8 bits
+};
+
+// XOR swizzle of 16-byte chunks: the eight threads of a quarter-warp, whose rows are ROWB bytes
+// apart, land in eight different 16-byte bank groups for every chunk index q.
+template <class C>
+__device__ __forceinline__ int swz(int row) {
+  return (C::CPR >= 8) ? (row & 7) : ((row >> 1) & 3);
+}
+template <class C>
+__device__ __forceinline__ int phys_chunk(int row, int q) {
+  return (row * C::CPR + q) ^ swz<C>(row);
+}
+
+// ------------------------------------------------------------------------------------------
+// cp.async
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ void cp_async16(void *smem, const void *gmem, int src_bytes) {
+  unsigned s = (unsigned)__cvta_generic_to_shared(smem);
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(s), "l"(gmem), "r"(src_bytes)
+               : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() {
+  asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory");
+}
+
+// Copy the rows of chunk `c` (tiles [c*TPC, (c+1)*TPC), clipped to n_tiles) into a swizzled stage.
+// Rows past the end of the tensor are zero-filled.
+template <class C>
+__device__ __forceinline__ void issue_chunk(const uint8_t *in, uint64_t n_tiles, uint64_t c, uint8_t *stage) {
+  const uint64_t tile0 = c * C::TPC;
+  const uint64_t rem = n_tiles - tile0;
+  const uint32_t valid_bytes = (uint32_t)(rem < (uint64_t)C::TPC ? rem : (uint64_t)C::TPC) * C::G * C::ESZ;
+  const uint8_t *src = in + tile0 * (uint64_t)(C::G * C::ESZ);
+#pragma unroll
+  for (int i = 0; i < C::CPR; ++i) {
+    const int ci = i * kThreads + (int)threadIdx.x;
+    const int row = ci / C::CPR;
+    const bool ok = (uint32_t)ci * 16u < valid_bytes;
+    cp_async16(stage + (size_t)(ci ^ swz<C>(row)) * 16, ok ? src + (size_t)ci * 16 : src, ok ? 16 : 0);
+  }
+}
+
+// Eight consecutive elements (oct `o`) of this thread's row, widened to binary32.
+template <class C>
+__device__ __forceinline__ void load_oct(const uint8_t *stage, int o, float (&v)[8]) {
+  const int row = (int)threadIdx.x;
+  if constexpr (C::BF16) {
+    const uint4 w = *reinterpret_cast<const uint4 *>(stage + (size_t)phys_chunk<C>(row, o) * 16);
+    const uint32_t u[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      v[2 * j] = __uint_as_float(u[j] << 16);
+      v[2 * j + 1] = __uint_as_float(u[j] & 0xffff0000u);
+    }
+  } else {
+    const float4 a = *reinterpret_cast<const float4 *>(stage + (size_t)phys_chunk<C>(row, 2 * o) * 16);
+    const float4 b = *reinterpret_cast<const float4 *>(stage + (size_t)phys_chunk<C>(row, 2 * o + 1) * 16);
+    v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w;
+    v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+  }
+}
+
+// One element of this thread's row (dynamic index), for the pivot.
+template <class C>
+__device__ __forceinline__ float load_elem(const uint8_t *stage, int k) {
+  const int row = (int)threadIdx.x;
+  constexpr int EPC = 16 / C::ESZ;
+  const uint8_t *p = stage + (size_t)phys_chunk<C>(row, k / EPC) * 16 + (size_t)(k % EPC) * C::ESZ;
+  if constexpr (C::BF16) return __uint_as_float((uint32_t)(*reinterpret_cast<const uint16_t *>(p)) << 16);
+  else return *reinterpret_cast<const float *>(p);
+}
+
+// ------------------------------------------------------------------------------------------
+// Arithmetic of Eq. 1-2 (binary32, fixed order; the library is compiled with -fmad=false so that
+// only the fused multiply-adds written here are fused)
+// ------------------------------------------------------------------------------------------
+
+// neighbours-first pairwise tree over 8 values
+__device__ __forceinline__ float tree8(const float (&v)[8]) {
+  const float a = v[0] + v[1], b = v[2] + v[3], c = v[4] + v[5], d = v[6] + v[7];
+  return (a + b) + (c + d);
+}
+template <int N>
+__device__ __forceinline__ float tree(float (&t)[N]) {
+#pragma unroll
+  for (int h = 1; h < N; h *= 2)
+#pragma unroll
+    for (int i = 0; i + h < N; i += 2 * h) t[i] = t[i] + t[i + h];
+  return t[0];
+}
+
+// log2 of a positive normal number: exponent + u*Q(u), u = mantissa - 1, Q of degree 5.
+__device__ __forceinline__ float lg2_poly(float x) {
+  const uint32_t xi = __float_as_uint(x);
+  const float e = (float)((int)(xi >> 23) - 127);
+  const float u = __uint_as_float((xi & 0x007fffffu) | 0x3f800000u) - 1.0f;
+  float q = -0x1.a762d6p-6f;
+  q = __fmaf_rn(q, u, 0x1.f2e252p-4f);
+  q = __fmaf_rn(q, u, -0x1.1c9334p-2f);
+  q = __fmaf_rn(q, u, 0x1.d487c6p-2f);
+  q = __fmaf_rn(q, u, -0x1.6fb0bcp-1f);
+  q = __fmaf_rn(q, u, 0x1.714aa0p+0f);
+  return __fmaf_rn(u, q, e);
+}
+
+// Entropy score of the tile this thread (pair) owns: -sum p log2(p + varsigma), p = |a| / (L1 + eps).
+template <class C>
+__device__ __forceinline__ float tile_score(const uint8_t *stage, float eps_l1, float eps_log) {
+  float part[C::NOCT];
+#pragma unroll
+  for (int o = 0; o < C::NOCT; ++o) {
+    float v[8];
+    load_oct<C>(stage, o, v);
+#pragma unroll
+    for (int k = 0; k < 8; ++k) v[k] = fabsf(v[k]);
+    part[o] = tree8(v);
+  }
+  float L1 = tree<C::NOCT>(part);
+  if constexpr (C::LPT == 2) L1 = L1 + __shfl_xor_sync(kFull, L1, 1);
+  const float inv = __fdiv_rn(1.0f, L1 + eps_l1);
+#pragma unroll
+  for (int o = 0; o < C::NOCT; ++o) {
+    float v[8];
+    load_oct<C>(stage, o, v);
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+      const float p = fabsf(v[k]) * inv;
+      v[k] = p * lg2_poly(p + eps_log);
+    }
+    part[o] = tree8(v);
+  }
+  float S = tree<C::NOCT>(part);
+  if constexpr (C::LPT == 2) S = S + __shfl_xor_sync(kFull, S, 1);
+  return 0.0f - S;
+}
+
+// Order-preserving map binary32 -> uint32, and the 64-bit ranking key (score first, then the
+// lower tile index wins): larger key = earlier in the ranking of Sec. 3.2.
+__device__ __forceinline__ uint32_t score_key32(float s) {
+  const uint32_t u = __float_as_uint(s);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ uint64_t rank_key(float s, uint32_t idx_in_group) {
+  return ((uint64_t)score_key32(s) << 32) | (uint64_t)(0xffffffffu - idx_in_group);
+}
+__device__ __forceinline__ uint32_t score_bin(float s) {
+  float t = fmaxf(s, 0.0f) * kBinScale;
+  t = fminf(t, (float)(kBins - 1));
+  return (uint32_t)t;   // truncation: monotone non-decreasing in s
+}
+
+// ------------------------------------------------------------------------------------------
+// Eq. 3-4 and the quantiser on a register-resident row
+// ------------------------------------------------------------------------------------------
+
+// In-thread butterfly (strides 1 .. EPT/2), neighbours first.
+template <int N>
+__device__ __forceinline__ void butterfly(float (&x)[N]) {
+#pragma unroll
+  for (int h = 1; h < N; h *= 2)
+#pragma unroll
+    for (int i = 0; i < N; ++i)
+      if (!(i & h)) {
+        const float a = x[i], b = x[i + h];
+        x[i] = a + b;
+        x[i + h] = a - b;
+      }
+}
+
+template <class C>
+__device__ __forceinline__ void hadamard_scaled(float (&x)[C::EPT]) {
+  butterfly<C::EPT>(x);
+  if constexpr (C::LPT == 2) {
+    const bool upper = threadIdx.x & 1;
+#pragma unroll
+    for (int k = 0; k < C::EPT; ++k) {
+      const float p = __shfl_xor_sync(kFull, x[k], 1);
+      x[k] = upper ? (p - x[k]) : (x[k] + p);
+    }
+  }
+  constexpr float c = (C::G == 32) ? 0.17677669529663687f : (C::G == 64) ? 0.125f : 0.08838834764831845f;
+#pragma unroll
+  for (int k = 0; k < C::EPT; ++k) x[k] = x[k] * c;
+}
+
+// Little-endian bit stream of N codes of W bits into N*W/32 words (all indices static).
+template <int W, int N>
+__device__ __forceinline__ void pack_words(const uint32_t (&c)[N], uint32_t *w) {
+#pragma unroll
+  for (int j = 0; j < N * W / 32; ++j) w[j] = 0;
+#pragma unroll
+  for (int k = 0; k < N; ++k) {
+    const int bit = k * W, j = bit >> 5, s = bit & 31;
+    w[j] |= c[k] << s;
+    if (s + W > 32) w[j + 1] |= c[k] >> (32 - s);
+  }
+}
+template <int W, int N>
+__device__ __forceinline__ void unpack_words(const uint32_t *w, uint32_t (&c)[N]) {
+#pragma unroll
+  for (int k = 0; k < N; ++k) {
+    const int bit = k * W, j = bit >> 5, s = bit & 31;
+    uint32_t v = w[j] >> s;
+    if (s + W > 32) v |= w[j + 1] << (32 - s);
+    c[k] = v & ((1u << W) - 1u);
+  }
+}
+
+}  // namespace tahq

@@ -1,0 +1,177 @@
+"""Parity of the CUDA path with the CPU oracle, through the C ABI, on the same seeded inputs.
+
+Bar: header, bit map, pivot bytes, binary16 scale/zero, offsets and sizes bit-exact; codes bit-exact
+(the kernels evaluate the oracle's binary32 expressions in the same order); decoded tensors equal."""
+import numpy as np
+import pytest
+import torch
+
+import oracle as O
+from paper_2506_01352_b200 import binding as T
+from paper_2506_01352_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+
+def oparams(p: T.Params) -> O.Params:
+    return O.Params(tokens=p.tokens, hidden=p.hidden, dtype=p.dtype, group_tokens=p.group_tokens, tile=p.tile,
+                    budget_millibits=p.budget_millibits, tau=p.tau, eps_l1=p.eps_l1, eps_log=p.eps_log,
+                    eps_ratio=p.eps_ratio, rounding=p.rounding, seed=p.seed)
+
+
+def sections(p: T.Params, buf: np.ndarray):
+    L = T.packed_layout(p)
+    n = L["n_tiles"]
+    return {
+        "header": buf[:128],
+        "bitmap": buf[L["off_bitmap"]:L["off_scale_zero"]],
+        "scale_zero": buf[L["off_scale_zero"]:L["off_pivot"]],
+        "pivot": buf[L["off_pivot"]:L["off_payload"]],
+        "payload": buf[L["off_payload"]:L["total_bytes"]],
+    }
+
+
+def check_encode(p: T.Params, x: torch.Tensor):
+    ws = T.alloc_workspace(p, x.device)
+    packed = T.alloc_packed(p, x.device)
+    packed.fill_(0xA5)                       # every byte must be overwritten
+    T.encode(p, x, packed=packed, ws=ws)
+    torch.cuda.synchronize()
+    assert T.device_status(ws) == 0
+    got = packed.cpu().numpy()
+    want = O.encode(oparams(p), synth.to_host_array(x))
+    assert got.size == want.size
+    gs, ws_ = sections(p, got), sections(p, want)
+    for name in ("header", "bitmap", "pivot", "scale_zero", "payload"):
+        if not np.array_equal(gs[name], ws_[name]):
+            bad = np.flatnonzero(gs[name] != ws_[name])
+            raise AssertionError(f"{name}: {bad.size} differing bytes, first at {bad[:8]}")
+    return packed, want, ws
+
+
+def check_decode(p: T.Params, packed: torch.Tensor, want_packed: np.ndarray, ws):
+    out = torch.full((p.tokens, p.hidden), float("nan"), device=packed.device,
+                     dtype=torch.float32 if p.dtype == T.F32 else torch.bfloat16)
+    T.decode(p, packed, out=out, ws=ws)
+    torch.cuda.synchronize()
+    assert T.device_status(ws) == 0
+    got = synth.to_host_array(out)
+    want = O.decode(oparams(p), want_packed)
+    assert np.array_equal(got.view(np.uint32 if p.dtype == T.F32 else np.uint16),
+                          want.view(np.uint32 if p.dtype == T.F32 else np.uint16))
+
+
+@pytest.mark.parametrize("G", [32, 64, 128])
+@pytest.mark.parametrize("beta", [4000, 3800, 3000, 2200, 6000, 8000, 7500])
+def test_c1_tiny(G, beta):
+    x = synth.make("c1_tiny", device="cuda")
+    p = T.params_for(x, group_tokens=64, tile=G, budget_millibits=beta)
+    packed, want, ws = check_encode(p, x)
+    check_decode(p, packed, want, ws)
+
+
+@pytest.mark.parametrize("G", [32, 64, 128])
+def test_c1_tiny_bf16(G):
+    x = synth.make("c1_tiny", device="cuda", microbatch=1).to(torch.bfloat16)
+    p = T.params_for(x, group_tokens=64, tile=G, budget_millibits=3500)
+    packed, want, ws = check_encode(p, x)
+    check_decode(p, packed, want, ws)
+
+
+@pytest.mark.parametrize("variant", [0, 1])
+@pytest.mark.parametrize("beta", [3000, 3800, 4000])
+def test_c2_gpt2_small(variant, beta):
+    x = synth.make("c2_gpt2s", variant=variant, device="cuda")
+    p = T.params_for(x, group_tokens=1024, tile=64, budget_millibits=beta)
+    packed, want, ws = check_encode(p, x)
+    check_decode(p, packed, want, ws)
+
+
+@pytest.mark.parametrize("beta", [3000, 3500, 3800, 4000])
+def test_c3_llama7b(beta):
+    x = synth.make("c3_llama7b", device="cuda")
+    p = T.params_for(x, group_tokens=2048, tile=64, budget_millibits=beta)
+    packed, want, ws = check_encode(p, x)
+    check_decode(p, packed, want, ws)
+
+
+@pytest.mark.parametrize("G,beta", [(32, 3000), (64, 3000), (128, 3000), (64, 3500)])
+def test_c4_llama13b(G, beta):
+    x = synth.make("c4_llama13b", device="cuda")
+    p = T.params_for(x, group_tokens=2048, tile=G, budget_millibits=beta)
+    packed, want, ws = check_encode(p, x)
+    check_decode(p, packed, want, ws)
+
+
+@pytest.mark.parametrize("shape,S,G", [((1, 64), 0, 64), ((1, 32), 1, 32), ((3, 128), 3, 128), ((7, 96), 7, 32),
+                                       ((300, 192), 100, 64), ((513, 640), 171, 128), ((1000, 64), 8, 64)])
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_ragged_and_degenerate_shapes(shape, S, G, dtype):
+    g = torch.Generator(device="cuda").manual_seed(shape[0] * 1000 + shape[1])
+    x = torch.randn(*shape, generator=g, device="cuda") * torch.randn(shape[0], 1, generator=g, device="cuda").exp()
+    x[:, ::37] *= 25
+    x = x.to(dtype)
+    for beta in (3800, 3000, 2500):
+        p = T.params_for(x, group_tokens=S, tile=G, budget_millibits=beta)
+        packed, want, ws = check_encode(p, x)
+        check_decode(p, packed, want, ws)
+
+
+@pytest.mark.parametrize("kind", ["zeros", "constant", "one_hot", "ties", "tau0", "tauinf", "huge"])
+def test_degenerate_values(kind):
+    T_, C_ = 256, 512
+    kw = {}
+    if kind == "zeros":
+        x = torch.zeros(T_, C_, device="cuda")
+    elif kind == "constant":
+        x = torch.full((T_, C_), 3.14159, device="cuda")        # every score ties: index order decides
+    elif kind == "one_hot":
+        x = torch.zeros(T_, C_, device="cuda")
+        x[:, 5::64] = torch.arange(1, T_ + 1, device="cuda", dtype=torch.float32)[:, None]
+    elif kind == "ties":
+        x = torch.randint(-2, 3, (T_, C_), device="cuda", generator=torch.Generator("cuda").manual_seed(1)).float()
+    elif kind == "huge":
+        x = torch.randn(T_, C_, device="cuda", generator=torch.Generator("cuda").manual_seed(2)) * 1e6
+    else:
+        x = synth.make("c1_tiny", device="cuda", microbatch=3).repeat(2, 2)
+        kw["tau"] = 0.0 if kind == "tau0" else float("inf")
+    for beta in (3800, 4000):
+        p = T.params_for(x, group_tokens=64, tile=64, budget_millibits=beta, **kw)
+        packed, want, ws = check_encode(p, x)
+        check_decode(p, packed, want, ws)
+
+
+def test_decode_refuses_a_foreign_buffer():
+    x = synth.make("c1_tiny", device="cuda")
+    p = T.params_for(x, group_tokens=64, budget_millibits=3800)
+    ws = T.alloc_workspace(p)
+    packed = T.encode(p, x, ws=ws)
+    out = torch.full_like(x, 7.0)
+    p2 = T.params_for(x, group_tokens=64, budget_millibits=3800, tau=3.0)
+    T.decode(p2, packed, out=out, ws=ws)
+    torch.cuda.synchronize()
+    assert T.device_status(ws) & T.DEV_BAD_HEADER
+    assert bool((out == 7.0).all())                              # output untouched
+    bad = packed.clone()
+    L = T.packed_layout(p)
+    bad[L["off_bitmap"]] ^= 0xFF                                 # bit-map population no longer matches
+    T.decode(p, bad, out=out, ws=ws)
+    torch.cuda.synchronize()
+    assert T.device_status(ws) & T.DEV_BAD_BITMAP
+    assert bool((out == 7.0).all())
+
+
+def test_deterministic_and_stream_ordered():
+    x = synth.make("c2_gpt2s", device="cuda")
+    p = T.params_for(x, group_tokens=1024, budget_millibits=3800)
+    s = torch.cuda.Stream()
+    ws = T.alloc_workspace(p)
+    with torch.cuda.stream(s):
+        a = T.encode(p, x, ws=ws, stream=s).clone()
+        b = T.encode(p, x, ws=ws, stream=s).clone()
+        y = T.decode(p, b, ws=ws, stream=s)
+    s.synchronize()
+    assert torch.equal(a, b)
+    assert T.last_launch_count() > 0
+    rel = ((y - x).double().pow(2).sum() / x.double().pow(2).sum()).item()
+    assert rel < 0.05

@@ -1,0 +1,71 @@
+"""Host-only checks of the C-ABI library (no GPU needed): it builds, loads, exports every symbol the
+header declares, and its size/layout functions agree with the oracle's independent arithmetic."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+import oracle as O
+from paper_2506_01352_b200 import binding as T
+from paper_2506_01352_b200 import build as B
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module", autouse=True)
+def built():
+    B.build()
+
+
+def test_every_declared_symbol_is_exported():
+    hdr = open(os.path.join(ROOT, "include", "tahq.h")).read()
+    hdr = re.sub(r"/\*.*?\*/", "", hdr, flags=re.S)
+    declared = set(re.findall(r"\b(tahq_[a-z0-9_]+)\s*\(", hdr))
+    assert {"tahq_encode", "tahq_decode", "tahq_packed_bound", "tahq_workspace_bound"} <= declared
+    lib = C.CDLL(B.LIB)
+    for name in sorted(declared):
+        assert hasattr(lib, name), f"{name} is declared in include/tahq.h but not exported"
+    assert declared == set(T.EXPORTS)
+
+
+CASES = [
+    dict(tokens=128, hidden=256, group_tokens=64, tile=64, budget_millibits=3800),
+    dict(tokens=128, hidden=256, group_tokens=64, tile=32, budget_millibits=4000),
+    dict(tokens=8192, hidden=768, group_tokens=1024, tile=64, budget_millibits=3000),
+    dict(tokens=8192, hidden=4096, dtype=1, group_tokens=2048, tile=64, budget_millibits=3500),
+    dict(tokens=16384, hidden=5120, group_tokens=2048, tile=128, budget_millibits=3000),
+    dict(tokens=65536, hidden=8192, dtype=1, group_tokens=4096, tile=64, budget_millibits=2200),
+    dict(tokens=77, hidden=96, group_tokens=11, tile=32, budget_millibits=7999),
+    dict(tokens=5, hidden=128, group_tokens=0, tile=128, budget_millibits=8000),
+]
+
+
+@pytest.mark.parametrize("kw", CASES)
+def test_layout_agrees_with_the_oracle(kw):
+    lt = T.packed_layout(T.Params(**kw))
+    lo = O.layout(O.Params(**kw))
+    assert lt == lo
+    assert T.packed_bound(T.Params(**kw)) == O.packed_bound(O.Params(**kw)) == lt["total_bytes"]
+    assert T.workspace_bound(T.Params(**kw)) >= 256
+
+
+def test_invalid_and_unsupported_parameters():
+    base = dict(tokens=128, hidden=256, group_tokens=64, tile=64, budget_millibits=3800)
+    for kw in [dict(tile=48), dict(hidden=100), dict(group_tokens=5), dict(budget_millibits=1999),
+               dict(budget_millibits=8001), dict(tile=256), dict(dtype=2), dict(tokens=0), dict(tau=-1.0),
+               dict(tile=16), dict(rounding=2)]:
+        p = T.Params(**{**base, **kw})
+        assert T.packed_bound(p) == 0 and T.workspace_bound(p) == 0
+        with pytest.raises(T.TahqError):
+            T.packed_layout(p)
+    # host-detectable errors come back before anything touches CUDA
+    p = T.Params(**base)
+    assert T.tahq_encode(p, 0, 0, 0, 0, 0, 0) == 1                       # null pointers
+    assert T.tahq_encode(p, 4096, 8192, 16, 12288, 1 << 30, 0) == 3      # packed buffer too small
+    assert T.tahq_encode(p, 4096, 8192, 1 << 30, 12288, 16, 0) == 3      # workspace too small
+    assert T.tahq_encode(p, 4100, 8192, 1 << 30, 12288, 1 << 30, 0) == 4  # misaligned input
+    assert T.tahq_decode(p, 8192, 1 << 30, 4104, 12288, 1 << 30, 0) == 4
+    bad = p.c(); bad.struct_size = 8
+    assert T.lib().tahq_packed_bound(C.byref(bad)) == 0
+    assert T.status_string(0) == "ok" and "small" in T.status_string(3)
