@@ -1,0 +1,348 @@
+#!/usr/bin/env python
+"""Benchmark of the TAH-Quant boundary codec on B200.
+
+A step is one pass of the whole hot path -- tahq_encode followed by tahq_decode -- over one
+synthetic LLaMA-7B-shaped boundary tensor (4x2048 tokens x 4096, bf16, tile 64, 3.8-bit budget).
+`value` is uncompressed GB/s of that round trip with inputs resident in HBM; `e2e` is the same
+metric with pinned-host inputs and outputs (copies inside the timed region).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "encode+decode GB/s (uncompressed bytes)"
+UNIT = "GB/s"
+L2_BYTES = 126e6
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch, from the ncu captures summarised under
+# profiles/ (same kernel, same workload); None until a capture exists for that kernel.
+NCU_TRAFFIC_BYTES = {}
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=40)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c3_llama7b")
+    ap.add_argument("--variant", type=int, default=0)
+    ap.add_argument("--budget", type=int, default=3800)
+    ap.add_argument("--tile", type=int, default=64)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    return ap.parse_args()
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            d = json.load(f)
+        return float(d["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._pump, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [t.strip() for t in ln.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for nm, v in zip(names, f[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def oracle_roundtrip_seconds(p_kw: dict, host_array, reps: int):
+    import oracle as O
+    po = O.Params(**p_kw)
+    cores = len(os.sched_getaffinity(0)) if hasattr(os, "sched_getaffinity") else (os.cpu_count() or 1)
+    O.set_threads(cores)
+    ts = []
+    for _ in range(reps):
+        t0 = time.perf_counter()
+        packed = O.encode(po, host_array)
+        O.decode(po, packed)
+        ts.append(time.perf_counter() - t0)
+    return ts, cores
+
+
+def run_reference(args):
+    """The reference arm: the CPU oracle, as it stands, on the host cores (rank 0 only)."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import torch
+    from paper_2506_01352_b200 import synth
+    w = synth.WORKLOADS[args.workload]
+    x = synth.make(args.workload, variant=args.variant, device="cpu")
+    h = synth.to_host_array(x)
+    kw = dict(tokens=w.tokens, hidden=w.hidden, dtype=1 if w.dtype == torch.bfloat16 else 0, group_tokens=w.seq,
+              tile=args.tile, budget_millibits=args.budget)
+    oracle_roundtrip_seconds(kw, h, max(1, min(args.warmup, 2)))
+    ts, cores = oracle_roundtrip_seconds(kw, h, args.steps)
+    sec = sum(ts) / len(ts)
+    val = h.nbytes / sec / 1e9
+    sample = f"whole {args.workload} tensor ({h.nbytes / 2**20:.0f} MiB), encode+decode, every step"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": args.workload, "tile": args.tile, "budget_millibits": args.budget,
+                   "tensor": f"{w.tokens}x{w.hidden} {str(w.dtype).split('.')[-1]}"},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2506_01352_b200 import binding as T
+    from paper_2506_01352_b200 import synth
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the codec has no CPU path")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    T.lib()
+
+    w = synth.WORKLOADS[args.workload]
+    n_sets = 4
+    # every rank encodes/decodes its own boundary tensors (one per pipeline-stage boundary): no collective
+    xs = [synth.make(args.workload, variant=args.variant, microbatch=rank * n_sets + i, device=dev)
+          for i in range(n_sets)]
+    p = T.params_for(xs[0], group_tokens=w.seq, tile=args.tile, budget_millibits=args.budget)
+    L = T.packed_layout(p)
+    in_bytes = xs[0].numel() * xs[0].element_size()
+    packed_bytes = L["total_bytes"]
+    packs = [T.alloc_packed(p, dev) for _ in range(n_sets)]
+    outs = [torch.empty_like(x) for x in xs]
+    ws = T.alloc_workspace(p, dev)
+    stream = torch.cuda.current_stream()
+    sh = int(stream.cuda_stream)
+    ptr = lambda t: t.data_ptr()
+
+    def enc(i):
+        rc = T.tahq_encode(p, ptr(xs[i]), ptr(packs[i]), packed_bytes, ptr(ws), ws.numel(), sh)
+        if rc:
+            raise T.TahqError(rc)
+        return T.last_launch_count()
+
+    def dec(i):
+        rc = T.tahq_decode(p, ptr(packs[i]), packed_bytes, ptr(outs[i]), ptr(ws), ws.numel(), sh)
+        if rc:
+            raise T.TahqError(rc)
+        return T.last_launch_count()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(fn, steps):
+        """fn(i) enqueues one step; returns max-over-ranks milliseconds for `steps` steps."""
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        e0.record(stream)
+        for i in range(steps):
+            fn(i)
+        e1.record(stream)
+        barrier()
+        ms = torch.tensor([e0.elapsed_time(e1)], device=dev)
+        if world > 1:
+            dist.all_reduce(ms, op=dist.ReduceOp.MAX)
+        return float(ms.item())
+
+    launches = [0]
+
+    def roundtrip(i):
+        k = i % n_sets
+        launches[0] += enc(k) + dec(k)
+
+    for i in range(max(3, args.warmup)):
+        roundtrip(i)
+    torch.cuda.synchronize()
+    assert T.device_status(ws) == 0
+
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    launches[0] = 0
+    ms_total = timed(roundtrip, args.steps)
+    gpu_launches = launches[0]
+    ms_enc = timed(lambda i: enc(i % n_sets), args.steps)
+    ms_dec = timed(lambda i: dec(i % n_sets), args.steps)
+    clocks = sampler.stop() if rank == 0 else {}
+
+    # per-kernel durations: the same steps once more with the library's event timing switched on
+    T.profile(True)
+    barrier()
+    for i in range(args.steps):
+        roundtrip(i)
+    torch.cuda.synchronize()
+    T.profile(False)
+    per = {}
+    for name, ms in T.profile_read():
+        n, t = per.get(name, (0, 0.0))
+        per[name] = (n + 1, t + ms)
+
+    # end to end: pinned host tensor -> device -> encode -> packed to host; packed from host -> decode -> host
+    hx = [x.cpu().pin_memory() for x in xs[:2]]
+    hp = [torch.empty(packed_bytes, dtype=torch.uint8).pin_memory() for _ in range(2)]
+    ho = [torch.empty_like(h).pin_memory() for h in hx]
+
+    def e2e_step(i):
+        k, j = i % n_sets, i % 2
+        xs[k].copy_(hx[j], non_blocking=True)
+        enc(k)
+        hp[j].copy_(packs[k], non_blocking=True)
+        packs[k].copy_(hp[j], non_blocking=True)
+        dec(k)
+        ho[j].copy_(outs[k], non_blocking=True)
+
+    for i in range(3):
+        e2e_step(i)
+    e2e_steps = max(3, min(args.steps, 20))
+    ms_e2e = timed(e2e_step, e2e_steps)
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peak, peak_kind = measured_peaks()
+    gb = lambda nbytes, ms, steps: nbytes * steps / (ms * 1e-3) / 1e9
+    value = gb(in_bytes * world, ms_total, args.steps)
+    # algorithmic bytes: encode reads the tensor once and writes the packed buffer;
+    # decode reads the packed buffer and writes the tensor
+    alg_dir = in_bytes + packed_bytes
+    n_tiles = L["n_tiles"]
+    alg_kernel = {
+        "stats": in_bytes + 4 * n_tiles,
+        "quant_pack": in_bytes + packed_bytes,
+        "decode": in_bytes + packed_bytes,
+    }
+    kern = []
+    tot_ms = sum(t for _, t in per.values()) or 1.0
+    for name, (n, t) in sorted(per.items(), key=lambda kv: -kv[1][1]):
+        kern.append({"kernel": name, "launches": n, "avg_us": 1e3 * t / n, "share": t / tot_ms})
+    dom = kern[0]["kernel"] if kern else None
+    roof = None
+    if dom in alg_kernel:
+        ach = alg_kernel[dom] / (per[dom][1] / per[dom][0] * 1e-3) / 1e9
+        roof = {"bound": "hbm", "kernel": dom, "achieved": ach, "peak": peak, "peak_kind": f"of {peak_kind}",
+                "unit": "GB/s", "frac": ach / peak,
+                "traffic": NCU_TRAFFIC_BYTES.get((dom, args.workload, args.budget, args.tile)),
+                "algorithmic_bytes_per_launch": alg_kernel[dom]}
+    path = {}
+    for nm, ms in (("encode", ms_enc), ("decode", ms_dec)):
+        a = gb(alg_dir, ms, args.steps)
+        path[nm] = {"uncompressed_GBps": gb(in_bytes, ms, args.steps), "us": 1e3 * ms / args.steps,
+                    "hbm_GBps": a, "frac_of_measured": a / peak, "frac_of_8TBps": a / 8000.0}
+    a = gb(2 * alg_dir, ms_total, args.steps)
+    path["roundtrip"] = {"uncompressed_GBps": value / world, "us": 1e3 * ms_total / args.steps, "hbm_GBps": a,
+                         "frac_of_measured": a / peak, "frac_of_8TBps": a / 8000.0}
+
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        kw = dict(tokens=w.tokens, hidden=w.hidden, dtype=p.dtype, group_tokens=w.seq, tile=args.tile,
+                  budget_millibits=args.budget)
+        h = synth.to_host_array(xs[0])
+        ts, cores = oracle_roundtrip_seconds(kw, h, 4)
+        sec = sum(ts[1:]) / len(ts[1:])
+        cpu = {"value": h.nbytes / sec / 1e9, "unit": UNIT, "cores": cores, "kind": "oracle",
+               "sample": f"whole {args.workload} tensor ({h.nbytes / 2**20:.0f} MiB), encode+decode, 3 timed passes"}
+
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(3, args.warmup), "ms_per_step": ms_total / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": args.workload, "tensor": f"{w.tokens}x{w.hidden} {str(w.dtype).split('.')[-1]}",
+                   "tile": args.tile, "budget_millibits": args.budget, "group_tokens": w.seq,
+                   "parallelism": f"{world} independent boundary tensors" if world > 1 else "1 GPU",
+                   "l2": f"rotating {n_sets} input/packed/output sets "
+                         f"({n_sets * (2 * in_bytes + packed_bytes) / 1e6:.0f} MB) > L2 ({L2_BYTES / 1e6:.0f} MB)"},
+        "e2e": {"value": gb(in_bytes * world, ms_e2e, e2e_steps), "unit": UNIT,
+                "h2d_bytes_per_step": in_bytes + packed_bytes, "d2h_bytes_per_step": in_bytes + packed_bytes,
+                "ms_per_step": ms_e2e / e2e_steps},
+        "gpu_launches": gpu_launches,
+        "clocks": clocks,
+        "roofline": roof,
+        "path": path,
+        "kernels": kern,
+        "cpu_baseline": cpu,
+    }
+    print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -136,6 +136,17 @@ const char *tahq_status_string(tahq_status s);
 /* Number of kernels the last tahq_encode / tahq_decode call of this thread enqueued. */
 int tahq_last_launch_count(void);
 
+/*
+ * Per-kernel timing for benchmarks (off by default; not thread-safe; the paper has no counterpart).
+ * tahq_profile(1) clears earlier records and makes every following kernel launch of the library be
+ * bracketed by two CUDA events on its stream; tahq_profile(0) stops recording.
+ * tahq_profile_read waits for the recorded events, writes up to max_records kernel names
+ * (32 bytes each, NUL-terminated, into `names`) and their durations in milliseconds (into `ms`),
+ * in launch order, clears the records and returns how many were written.  Host pointers.
+ */
+void tahq_profile(int enable);
+int tahq_profile_read(char *names, float *ms, int max_records);
+
 #ifdef __cplusplus
 }
 #endif

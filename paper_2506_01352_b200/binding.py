@@ -67,7 +67,7 @@ class TahqError(RuntimeError):
 
 
 EXPORTS = ["tahq_packed_bound", "tahq_packed_layout", "tahq_workspace_bound", "tahq_encode", "tahq_decode",
-           "tahq_status_string", "tahq_last_launch_count"]
+           "tahq_status_string", "tahq_last_launch_count", "tahq_profile", "tahq_profile_read"]
 
 _lib = None
 
@@ -94,6 +94,10 @@ def lib() -> C.CDLL:
         L.tahq_status_string.restype = C.c_char_p
         L.tahq_last_launch_count.argtypes = []
         L.tahq_last_launch_count.restype = C.c_int
+        L.tahq_profile.argtypes = [C.c_int]
+        L.tahq_profile.restype = None
+        L.tahq_profile_read.argtypes = [C.c_char_p, C.POINTER(C.c_float), C.c_int]
+        L.tahq_profile_read.restype = C.c_int
         _lib = L
     return _lib
 
@@ -122,6 +126,19 @@ def packed_layout(p: Params) -> dict:
 
 def last_launch_count() -> int:
     return int(lib().tahq_last_launch_count())
+
+
+def profile(enable: bool) -> None:
+    """Switch the library's per-kernel event timing on or off."""
+    lib().tahq_profile(1 if enable else 0)
+
+
+def profile_read(max_records: int = 65536):
+    """[(kernel name, milliseconds), ...] of the launches recorded since profile(True); synchronises."""
+    names = C.create_string_buffer(32 * max_records)
+    ms = (C.c_float * max_records)()
+    n = lib().tahq_profile_read(names, ms, max_records)
+    return [(names.raw[32 * i:32 * i + 32].split(b"\0")[0].decode(), float(ms[i])) for i in range(n)]
 
 
 def _stream_handle(stream) -> int:

@@ -4,12 +4,37 @@
 
 #include <atomic>
 #include <cstring>
+#include <vector>
 
 #include "tahq_kernels.cuh"
 
 namespace tahq {
 
 static thread_local int g_launches = 0;
+
+// Optional per-kernel timing (tahq_profile): every launch is bracketed by two events on its stream.
+struct ProfRec { const char *name; cudaEvent_t e0, e1; };
+static bool g_prof_on = false;
+static std::vector<ProfRec> g_prof;
+
+struct LaunchScope {
+  cudaStream_t st;
+  bool on;
+  LaunchScope(const char *name, cudaStream_t s) : st(s), on(g_prof_on) {
+    ++g_launches;
+    if (on) {
+      ProfRec r{name, nullptr, nullptr};
+      cudaEventCreate(&r.e0);
+      cudaEventCreate(&r.e1);
+      cudaEventRecord(r.e0, st);
+      g_prof.push_back(r);
+    }
+  }
+  ~LaunchScope() {
+    if (on) cudaEventRecord(g_prof.back().e1, st);
+  }
+};
+#define TAHQ_LAUNCH(name, st, ...) do { LaunchScope scope_(name, st); __VA_ARGS__; } while (0)
 
 struct Plan {
   tahq_layout L;
@@ -172,25 +197,24 @@ static tahq_status encode_t(const Plan &pl, const Args &a, cudaStream_t st) {
     const int occ = prepare(stats_kernel<C, NS>, smem, d, occ_stats);
     if (!occ) return TAHQ_ERR_CUDA;
     const uint64_t cap = (uint64_t)d.sms * occ;
-    stats_kernel<C, NS><<<(unsigned)(n_chunks < cap ? n_chunks : cap), kThreads, smem, st>>>(a);
-    ++g_launches;
+    TAHQ_LAUNCH("stats", st,
+                stats_kernel<C, NS><<<(unsigned)(n_chunks < cap ? n_chunks : cap), kThreads, smem, st>>>(a));
     if (!pl.direct) {
-      hist_kernel<<<(unsigned)(a.n_groups * a.cpg), kThreads, 0, st>>>(a);
-      gather_kernel<<<(unsigned)(a.n_groups * a.cpg), kThreads, 0, st>>>(a);
-      g_launches += 2;
+      TAHQ_LAUNCH("hist", st, hist_kernel<<<(unsigned)(a.n_groups * a.cpg), kThreads, 0, st>>>(a));
+      TAHQ_LAUNCH("gather", st, gather_kernel<<<(unsigned)(a.n_groups * a.cpg), kThreads, 0, st>>>(a));
     }
-    resolve_kernel<<<(unsigned)a.n_groups, kResolveThreads, 0, st>>>(a);
-    bitmap_kernel<<<(unsigned)((a.n_tiles + kThreads - 1) / kThreads), kThreads, 0, st>>>(a);
-    scan_kernel<<<1, kScanThreads, 0, st>>>(a.cnt128, pl.n128, ~0ull, a.status);
-    g_launches += 3;
+    TAHQ_LAUNCH("resolve", st, resolve_kernel<<<(unsigned)a.n_groups, kResolveThreads, 0, st>>>(a));
+    TAHQ_LAUNCH("bitmap", st,
+                bitmap_kernel<<<(unsigned)((a.n_tiles + kThreads - 1) / kThreads), kThreads, 0, st>>>(a));
+    TAHQ_LAUNCH("scan", st, scan_kernel<<<1, kScanThreads, 0, st>>>(a.cnt128, pl.n128, ~0ull, a.status));
   }
   constexpr int NQ = Stages<C>::QUANT;
   const int smem = NQ * C::STAGE_BYTES + C::MAX_PAY;
   const int occ = prepare(quant_pack_kernel<C, NQ>, smem, d, occ_quant);
   if (!occ) return TAHQ_ERR_CUDA;
   const uint64_t cap = (uint64_t)d.sms * occ;
-  quant_pack_kernel<C, NQ><<<(unsigned)(n_chunks < cap ? n_chunks : cap), kThreads, smem, st>>>(a);
-  ++g_launches;
+  TAHQ_LAUNCH("quant_pack", st,
+              quant_pack_kernel<C, NQ><<<(unsigned)(n_chunks < cap ? n_chunks : cap), kThreads, smem, st>>>(a));
   return cudaGetLastError() == cudaSuccess ? TAHQ_OK : TAHQ_ERR_CUDA;
 }
 
@@ -200,14 +224,15 @@ static tahq_status decode_t(const Plan &pl, const Args &a, cudaStream_t st) {
   if (!dev_info(&d)) return TAHQ_ERR_CUDA;
   const uint64_t n_chunks = (a.n_tiles + C::TPC - 1) / C::TPC;
   static std::atomic<int> occ_dec[64];
-  count_kernel<<<(unsigned)((pl.n128 + kThreads - 1) / kThreads), kThreads, 0, st>>>(a);
-  scan_kernel<<<1, kScanThreads, 0, st>>>(a.cnt128, pl.n128, pl.mixed ? a.n_groups * a.k_hi : ~0ull, a.status);
+  TAHQ_LAUNCH("count", st, count_kernel<<<(unsigned)((pl.n128 + kThreads - 1) / kThreads), kThreads, 0, st>>>(a));
+  TAHQ_LAUNCH("scan", st, scan_kernel<<<1, kScanThreads, 0, st>>>(a.cnt128, pl.n128,
+                                                                 pl.mixed ? a.n_groups * a.k_hi : ~0ull, a.status));
   const int smem = C::STAGE_BYTES;
   const int occ = prepare(decode_kernel<C>, smem, d, occ_dec);
   if (!occ) return TAHQ_ERR_CUDA;
   const uint64_t cap = (uint64_t)d.sms * occ * 8;
-  decode_kernel<C><<<(unsigned)(n_chunks < cap ? n_chunks : cap), kThreads, smem, st>>>(a);
-  g_launches += 3;
+  TAHQ_LAUNCH("decode", st,
+              decode_kernel<C><<<(unsigned)(n_chunks < cap ? n_chunks : cap), kThreads, smem, st>>>(a));
   return cudaGetLastError() == cudaSuccess ? TAHQ_OK : TAHQ_ERR_CUDA;
 }
 
@@ -297,5 +322,31 @@ const char *tahq_status_string(tahq_status s) {
 }
 
 int tahq_last_launch_count(void) { return g_launches; }
+
+void tahq_profile(int enable) {
+  g_prof_on = enable != 0;
+  if (g_prof_on) {
+    for (auto &r : g_prof) { cudaEventDestroy(r.e0); cudaEventDestroy(r.e1); }
+    g_prof.clear();
+  }
+}
+
+int tahq_profile_read(char *names, float *ms, int max_records) {
+  int n = 0;
+  for (auto &r : g_prof) {
+    if (n < max_records) {
+      cudaEventSynchronize(r.e1);
+      float t = 0.0f;
+      cudaEventElapsedTime(&t, r.e0, r.e1);
+      if (ms) ms[n] = t;
+      if (names) { std::strncpy(names + 32 * n, r.name, 31); names[32 * n + 31] = 0; }
+      ++n;
+    }
+    cudaEventDestroy(r.e0);
+    cudaEventDestroy(r.e1);
+  }
+  g_prof.clear();
+  return n;
+}
 
 }  // extern "C"
