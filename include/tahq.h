@@ -124,7 +124,10 @@ tahq_status tahq_encode(const tahq_params *p, const void *d_in, void *d_packed, 
  * (dtype): bit map -> widths and offsets, unpack, z + q*s, inverse Hadamard
  * and un-swap on flagged tiles, store (round-to-nearest-even for bf16).
  * The header inside d_packed must describe the same parameters; a mismatch is
- * reported through the device status word and the output is left untouched.
+ * reported through the device status word (TAHQ_DEV_BAD_HEADER) and the output
+ * is left untouched.  A bit map whose population does not match the payload
+ * size is reported as TAHQ_DEV_BAD_BITMAP; the output is then unspecified, and
+ * no byte outside the two buffers is read or written.
  * Errors as for tahq_encode (packed_bytes must be >= tahq_packed_bound()).
  */
 tahq_status tahq_decode(const tahq_params *p, const void *d_packed, size_t packed_bytes, void *d_out,

@@ -42,9 +42,8 @@ struct Plan {
   bool mixed;             // two widths in use (k_hi > 0)
   bool direct;            // small ranking groups: select straight from the scores
   uint32_t cpg, cand_cap;
-  uint64_t n128;
   // workspace offsets
-  uint64_t ws_ncand, ws_hist, ws_zero_end, ws_scores, ws_binsel, ws_theta, ws_cand, ws_cnt, ws_total;
+  uint64_t ws_flags, ws_ncand, ws_done, ws_hist, ws_zero_end, ws_scores, ws_theta, ws_cand, ws_total;
 };
 
 static uint64_t up(uint64_t x, uint64_t a) { return (x + a - 1) / a * a; }
@@ -82,24 +81,24 @@ static tahq_status make_plan(const tahq_params *p, Plan *pl) {
   if (p->rounding != 0) return TAHQ_ERR_UNSUPPORTED;
 
   pl->mixed = L.k_hi > 0;
-  pl->direct = L.tiles_per_group <= 16384;
+  pl->direct = L.tiles_per_group <= (uint64_t)kSortCap;
   pl->cpg = 1;
   pl->cand_cap = 0;
   if (pl->mixed && !pl->direct) {
-    uint64_t cpg = (L.tiles_per_group + 8191) / 8192;
-    pl->cpg = (uint32_t)(cpg > 128 ? 128 : cpg);
+    uint64_t cpg = (L.tiles_per_group + 16383) / 16384;
+    pl->cpg = (uint32_t)(cpg > 64 ? 64 : cpg);
     pl->cand_cap = (uint32_t)(L.tiles_per_group < 32768 ? L.tiles_per_group : 32768);
   }
-  pl->n128 = (L.n_tiles + 127) / 128;
+  const bool hist = pl->mixed && !pl->direct;
   uint64_t o = 256;                                         // status word and friends
-  pl->ws_ncand = o;  o = up(o + 4 * L.n_groups, 256);
-  pl->ws_hist = o;   o += (pl->mixed && !pl->direct) ? 4ull * kBins * L.n_groups : 0;
-  pl->ws_zero_end = o;                                      // [0, ws_zero_end) is cleared per call
+  pl->ws_flags = o;  o += 8ull * kMaxGrid;
+  pl->ws_ncand = o;  o = up(o + (hist ? 4 * L.n_groups : 0), 256);
+  pl->ws_done = o;   o = up(o + (hist ? 4 * L.n_groups : 0), 256);
+  pl->ws_hist = o;   o += hist ? 4ull * kBins * L.n_groups : 0;
+  pl->ws_zero_end = o;                                      // [0, ws_zero_end) is cleared by every encode
   pl->ws_scores = o; o = up(o + (pl->mixed ? 4 * L.n_tiles : 0), 256);
-  pl->ws_binsel = o; o = up(o + 8 * L.n_groups, 256);
-  pl->ws_theta = o;  o = up(o + 8 * L.n_groups, 256);
+  pl->ws_theta = o;  o = up(o + (pl->mixed ? 8 * L.n_groups : 0), 256);
   pl->ws_cand = o;   o = up(o + 8ull * pl->cand_cap * L.n_groups, 256);
-  pl->ws_cnt = o;    o = up(o + 4 * (pl->n128 + 2), 256);
   pl->ws_total = o;
   return TAHQ_OK;
 }
@@ -149,10 +148,10 @@ static void fill_args(const tahq_params *p, const Plan &pl, uint8_t *ws, Args *a
   a->ncand = reinterpret_cast<uint32_t *>(ws + pl.ws_ncand);
   a->hist = reinterpret_cast<uint32_t *>(ws + pl.ws_hist);
   a->scores = reinterpret_cast<float *>(ws + pl.ws_scores);
-  a->binsel = reinterpret_cast<uint2 *>(ws + pl.ws_binsel);
+  a->done = reinterpret_cast<uint32_t *>(ws + pl.ws_done);
+  a->flags = reinterpret_cast<unsigned long long *>(ws + pl.ws_flags);
   a->theta = reinterpret_cast<unsigned long long *>(ws + pl.ws_theta);
   a->cand = reinterpret_cast<unsigned long long *>(ws + pl.ws_cand);
-  a->cnt128 = reinterpret_cast<uint32_t *>(ws + pl.ws_cnt);
   a->cand_cap = pl.cand_cap;
   a->cpg = pl.cpg;
   a->direct = pl.direct;
@@ -182,39 +181,42 @@ static int prepare(K kernel, int smem, const DevInfo &d, std::atomic<int> *cache
 
 template <class C> struct Stages {
   static constexpr int STATS = (C::ROWB == 256) ? 2 : (C::ROWB == 128 ? 3 : 4);
-  static constexpr int QUANT = (C::ROWB == 256) ? 3 : (C::ROWB == 128 ? 3 : 4);
+  static constexpr int QUANT = (C::ROWB == 256) ? 2 : (C::ROWB == 128 ? 2 : 3);
 };
+
+// CTAs of a persistent tile kernel: every SM filled to the kernel's occupancy, never more than chunks.
+static unsigned persistent_grid(uint64_t n_chunks, const DevInfo &d, int occ) {
+  uint64_t cap = (uint64_t)d.sms * occ;
+  if (cap > (uint64_t)kMaxGrid) cap = kMaxGrid;
+  return (unsigned)(n_chunks < cap ? n_chunks : cap);
+}
 
 template <class C>
 static tahq_status encode_t(const Plan &pl, const Args &a, cudaStream_t st) {
   DevInfo d;
   if (!dev_info(&d)) return TAHQ_ERR_CUDA;
   const uint64_t n_chunks = (a.n_tiles + C::TPC - 1) / C::TPC;
-  static std::atomic<int> occ_stats[64], occ_quant[64];
+  static std::atomic<int> occ_stats[64], occ_quant[64], sel_ready[64];
   if (pl.mixed) {
     constexpr int NS = Stages<C>::STATS;
     const int smem = NS * C::STAGE_BYTES;
     const int occ = prepare(stats_kernel<C, NS>, smem, d, occ_stats);
     if (!occ) return TAHQ_ERR_CUDA;
-    const uint64_t cap = (uint64_t)d.sms * occ;
-    TAHQ_LAUNCH("stats", st,
-                stats_kernel<C, NS><<<(unsigned)(n_chunks < cap ? n_chunks : cap), kThreads, smem, st>>>(a));
-    if (!pl.direct) {
-      TAHQ_LAUNCH("hist", st, hist_kernel<<<(unsigned)(a.n_groups * a.cpg), kThreads, 0, st>>>(a));
-      TAHQ_LAUNCH("gather", st, gather_kernel<<<(unsigned)(a.n_groups * a.cpg), kThreads, 0, st>>>(a));
+    TAHQ_LAUNCH("stats", st, stats_kernel<C, NS><<<persistent_grid(n_chunks, d, occ), kThreads, smem, st>>>(a));
+    const int sel_smem = kSortCap * 8;
+    if (!sel_ready[d.dev & 63].load(std::memory_order_acquire)) {
+      if (cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, sel_smem) != cudaSuccess)
+        return TAHQ_ERR_CUDA;
+      sel_ready[d.dev & 63].store(1, std::memory_order_release);
     }
-    TAHQ_LAUNCH("resolve", st, resolve_kernel<<<(unsigned)a.n_groups, kResolveThreads, 0, st>>>(a));
-    TAHQ_LAUNCH("bitmap", st,
-                bitmap_kernel<<<(unsigned)((a.n_tiles + kThreads - 1) / kThreads), kThreads, 0, st>>>(a));
-    TAHQ_LAUNCH("scan", st, scan_kernel<<<1, kScanThreads, 0, st>>>(a.cnt128, pl.n128, ~0ull, a.status));
+    TAHQ_LAUNCH("select", st, select_kernel<<<(unsigned)(a.n_groups * a.cpg), kSelThreads, sel_smem, st>>>(a));
   }
   constexpr int NQ = Stages<C>::QUANT;
   const int smem = NQ * C::STAGE_BYTES + C::MAX_PAY;
   const int occ = prepare(quant_pack_kernel<C, NQ>, smem, d, occ_quant);
   if (!occ) return TAHQ_ERR_CUDA;
-  const uint64_t cap = (uint64_t)d.sms * occ;
   TAHQ_LAUNCH("quant_pack", st,
-              quant_pack_kernel<C, NQ><<<(unsigned)(n_chunks < cap ? n_chunks : cap), kThreads, smem, st>>>(a));
+              quant_pack_kernel<C, NQ><<<persistent_grid(n_chunks, d, occ), kThreads, smem, st>>>(a));
   return cudaGetLastError() == cudaSuccess ? TAHQ_OK : TAHQ_ERR_CUDA;
 }
 
@@ -224,15 +226,11 @@ static tahq_status decode_t(const Plan &pl, const Args &a, cudaStream_t st) {
   if (!dev_info(&d)) return TAHQ_ERR_CUDA;
   const uint64_t n_chunks = (a.n_tiles + C::TPC - 1) / C::TPC;
   static std::atomic<int> occ_dec[64];
-  TAHQ_LAUNCH("count", st, count_kernel<<<(unsigned)((pl.n128 + kThreads - 1) / kThreads), kThreads, 0, st>>>(a));
-  TAHQ_LAUNCH("scan", st, scan_kernel<<<1, kScanThreads, 0, st>>>(a.cnt128, pl.n128,
-                                                                 pl.mixed ? a.n_groups * a.k_hi : ~0ull, a.status));
   const int smem = C::STAGE_BYTES;
   const int occ = prepare(decode_kernel<C>, smem, d, occ_dec);
   if (!occ) return TAHQ_ERR_CUDA;
-  const uint64_t cap = (uint64_t)d.sms * occ * 8;
-  TAHQ_LAUNCH("decode", st,
-              decode_kernel<C><<<(unsigned)(n_chunks < cap ? n_chunks : cap), kThreads, smem, st>>>(a));
+  (void)pl;
+  TAHQ_LAUNCH("decode", st, decode_kernel<C><<<persistent_grid(n_chunks, d, occ), kThreads, smem, st>>>(a));
   return cudaGetLastError() == cudaSuccess ? TAHQ_OK : TAHQ_ERR_CUDA;
 }
 
@@ -300,7 +298,7 @@ tahq_status tahq_decode(const tahq_params *p, const void *d_packed, size_t packe
   fill_args(p, pl, static_cast<uint8_t *>(d_ws), &a);
   a.packed = const_cast<uint8_t *>(static_cast<const uint8_t *>(d_packed));
   a.out = static_cast<uint8_t *>(d_out);
-  if (cudaMemsetAsync(d_ws, 0, 256, st) != cudaSuccess) return TAHQ_ERR_CUDA;
+  if (cudaMemsetAsync(d_ws, 0, pl.ws_ncand, st) != cudaSuccess) return TAHQ_ERR_CUDA;   // status + flags
   const bool bf = p->dtype == TAHQ_BF16;
   switch (p->tile) {
     case 32: return bf ? decode_t<Cfg<32, true>>(pl, a, st) : decode_t<Cfg<32, false>>(pl, a, st);

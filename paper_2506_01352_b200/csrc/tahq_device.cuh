@@ -81,8 +81,7 @@ __device__ __forceinline__ void issue_chunk(const uint8_t *in, uint64_t n_tiles,
 
 // Eight consecutive elements (oct `o`) of this thread's row, widened to binary32.
 template <class C>
-__device__ __forceinline__ void load_oct(const uint8_t *stage, int o, float (&v)[8]) {
-  const int row = (int)threadIdx.x;
+__device__ __forceinline__ void load_oct(const uint8_t *stage, int row, int o, float (&v)[8]) {
   if constexpr (C::BF16) {
     const uint4 w = *reinterpret_cast<const uint4 *>(stage + (size_t)phys_chunk<C>(row, o) * 16);
     const uint32_t u[4] = {w.x, w.y, w.z, w.w};
@@ -101,8 +100,7 @@ __device__ __forceinline__ void load_oct(const uint8_t *stage, int o, float (&v)
 
 // One element of this thread's row (dynamic index), for the pivot.
 template <class C>
-__device__ __forceinline__ float load_elem(const uint8_t *stage, int k) {
-  const int row = (int)threadIdx.x;
+__device__ __forceinline__ float load_elem(const uint8_t *stage, int row, int k) {
   constexpr int EPC = 16 / C::ESZ;
   const uint8_t *p = stage + (size_t)phys_chunk<C>(row, k / EPC) * 16 + (size_t)(k % EPC) * C::ESZ;
   if constexpr (C::BF16) return __uint_as_float((uint32_t)(*reinterpret_cast<const uint16_t *>(p)) << 16);
@@ -149,7 +147,7 @@ __device__ __forceinline__ float tile_score(const uint8_t *stage, float eps_l1, 
 #pragma unroll
   for (int o = 0; o < C::NOCT; ++o) {
     float v[8];
-    load_oct<C>(stage, o, v);
+    load_oct<C>(stage, (int)threadIdx.x, o, v);
 #pragma unroll
     for (int k = 0; k < 8; ++k) v[k] = fabsf(v[k]);
     part[o] = tree8(v);
@@ -160,7 +158,7 @@ __device__ __forceinline__ float tile_score(const uint8_t *stage, float eps_l1, 
 #pragma unroll
   for (int o = 0; o < C::NOCT; ++o) {
     float v[8];
-    load_oct<C>(stage, o, v);
+    load_oct<C>(stage, (int)threadIdx.x, o, v);
 #pragma unroll
     for (int k = 0; k < 8; ++k) {
       const float p = fabsf(v[k]) * inv;
@@ -242,6 +240,160 @@ __device__ __forceinline__ void unpack_words(const uint32_t *w, uint32_t (&c)[N]
     uint32_t v = w[j] >> s;
     if (s + W > 32) v |= w[j + 1] << (32 - s);
     c[k] = v & ((1u << W) - 1u);
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// Stable counting sort of the 256 threads of a CTA by a 2-bit class, so that the warps that go
+// on are (nearly) uniform in (transformed?, higher width?) and neither the Hadamard butterfly nor
+// the width-specific packing runs divergent.  Two __syncthreads inside.
+// ------------------------------------------------------------------------------------------
+struct ClassSort {
+  int src;   // which thread's tile this thread processes from now on
+  int cls;   // class of that tile
+};
+__device__ __forceinline__ ClassSort sort_by_class(int cls, uint8_t *s_perm, uint2 *s_cnt) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const unsigned b1 = __ballot_sync(kFull, cls & 1), b2 = __ballot_sync(kFull, cls & 2);
+  const unsigned m0 = ~b1 & ~b2, m1 = b1 & ~b2, m2 = ~b1 & b2, m3 = b1 & b2;
+  if (lane == 0) s_cnt[warp] = make_uint2(__popc(m0) | (__popc(m1) << 16), __popc(m2) | (__popc(m3) << 16));
+  __syncthreads();
+  uint32_t tot_lo = 0, tot_hi = 0, bef_lo = 0, bef_hi = 0;   // two 16-bit counters per word
+#pragma unroll
+  for (int w = 0; w < kThreads / 32; ++w) {
+    const uint2 c = s_cnt[w];
+    tot_lo += c.x; tot_hi += c.y;
+    bef_lo += (w < warp) ? c.x : 0u;
+    bef_hi += (w < warp) ? c.y : 0u;
+  }
+  const int base1 = tot_lo & 0xffff, base2 = base1 + (tot_lo >> 16), base3 = base2 + (tot_hi & 0xffff);
+  const unsigned mine = (cls == 0) ? m0 : (cls == 1) ? m1 : (cls == 2) ? m2 : m3;
+  const int before = (cls == 0) ? (bef_lo & 0xffff) : (cls == 1) ? (bef_lo >> 16) : (cls == 2) ? (bef_hi & 0xffff)
+                                                                                               : (bef_hi >> 16);
+  const int base = (cls == 0) ? 0 : (cls == 1) ? base1 : (cls == 2) ? base2 : base3;
+  s_perm[base + before + __popc(mine & ((1u << lane) - 1u))] = (uint8_t)threadIdx.x;
+  __syncthreads();
+  ClassSort r;
+  r.src = s_perm[threadIdx.x];
+  const int t = threadIdx.x;
+  r.cls = (t >= base1) + (t >= base2) + (t >= base3);
+  return r;
+}
+
+// ------------------------------------------------------------------------------------------
+// bf16 pairs handled in their packed form (sm_100a: packed bf16 min/max run on the ALU pipe, one
+// instruction per two elements; a bf16 operand can feed an fp32 add on the FMA pipe directly)
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t bf2_max_abs(uint32_t a, uint32_t b) {   // magnitudes; sign bits are garbage
+  uint32_t d;
+  asm("max.xorsign.abs.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+  return d;
+}
+__device__ __forceinline__ uint32_t bf2_min_abs(uint32_t a, uint32_t b) {
+  uint32_t d;
+  asm("min.xorsign.abs.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+  return d;
+}
+__device__ __forceinline__ uint32_t bf2_max(uint32_t a, uint32_t b) {
+  uint32_t d;
+  asm("max.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+  return d;
+}
+__device__ __forceinline__ uint32_t bf2_min(uint32_t a, uint32_t b) {
+  uint32_t d;
+  asm("min.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+  return d;
+}
+// (lo + c, hi + c) in binary32 for the two bf16 halves of w: the widening is exact, so this equals
+// widening first and adding afterwards; with c = -0.0f it is the widening itself.
+__device__ __forceinline__ void bf2_add_f32(uint32_t w, float c, float &lo, float &hi) {
+  asm("{\n\t.reg .b16 l, h;\n\tmov.b32 {l, h}, %2;\n\tadd.rn.f32.bf16 %0, l, %3;\n\tadd.rn.f32.bf16 %1, h, %3;\n\t}"
+      : "=f"(lo), "=f"(hi)
+      : "r"(w), "f"(c));
+}
+
+// Largest and second-largest magnitude of a row (Eq. 3), no index.
+template <class C>
+__device__ __forceinline__ void row_top2(const uint8_t *stage, int row, float &a1, float &a2) {
+  if constexpr (C::BF16) {
+    uint32_t p1 = 0, p2 = 0, q1 = 0, q2 = 0;   // two independent (largest, second) pairs per 16-bit lane
+#pragma unroll
+    for (int q = 0; q < C::CPR; ++q) {
+      const uint4 w = *reinterpret_cast<const uint4 *>(stage + (size_t)phys_chunk<C>(row, q) * 16);
+      p2 = bf2_max_abs(p2, bf2_min_abs(p1, w.x)); p1 = bf2_max_abs(p1, w.x);
+      q2 = bf2_max_abs(q2, bf2_min_abs(q1, w.y)); q1 = bf2_max_abs(q1, w.y);
+      p2 = bf2_max_abs(p2, bf2_min_abs(p1, w.z)); p1 = bf2_max_abs(p1, w.z);
+      q2 = bf2_max_abs(q2, bf2_min_abs(q1, w.w)); q1 = bf2_max_abs(q1, w.w);
+    }
+    const uint32_t m1 = bf2_max_abs(p1, q1) & 0x7fff7fffu;
+    const uint32_t m2 = bf2_max_abs(bf2_min_abs(p1, q1), bf2_max_abs(p2, q2)) & 0x7fff7fffu;
+    const uint32_t e1 = m1 & 0xffffu, o1 = m1 >> 16, e2 = m2 & 0xffffu, o2 = m2 >> 16;
+    a1 = __uint_as_float(max(e1, o1) << 16);
+    a2 = __uint_as_float(max(min(e1, o1), max(e2, o2)) << 16);
+  } else {
+    float p1 = 0.0f, p2 = 0.0f, q1 = 0.0f, q2 = 0.0f;
+#pragma unroll
+    for (int q = 0; q < C::CPR; ++q) {
+      const float4 v = *reinterpret_cast<const float4 *>(stage + (size_t)phys_chunk<C>(row, q) * 16);
+      const float t0 = fabsf(v.x), t1 = fabsf(v.y), t2 = fabsf(v.z), t3 = fabsf(v.w);
+      p2 = fmaxf(p2, fminf(p1, t0)); p1 = fmaxf(p1, t0);
+      q2 = fmaxf(q2, fminf(q1, t1)); q1 = fmaxf(q1, t1);
+      p2 = fmaxf(p2, fminf(p1, t2)); p1 = fmaxf(p1, t2);
+      q2 = fmaxf(q2, fminf(q1, t3)); q1 = fmaxf(q1, t3);
+    }
+    a1 = fmaxf(p1, q1);
+    a2 = fmaxf(fminf(p1, q1), fmaxf(p2, q2));
+  }
+}
+
+__host__ __device__ constexpr uint64_t group_ones(int W, int GS) {
+  uint64_t v = 0;
+  for (int i = 0; i < GS; ++i) v |= 1ull << (W * i);
+  return v;
+}
+
+// Codes -> little-endian bit stream.  t[k] = q_k + 1.5*2^23 as binary32 (the rounding trick leaves
+// the integer code in the low mantissa bits); groups of codes are combined by multiply-adds on the
+// raw bit patterns and the constant's contribution is subtracted once per group.
+template <int W, int N, class F>
+__device__ __forceinline__ void pack_magic(F &&t, uint32_t *w) {
+  constexpr int GS = (W <= 4) ? 8 : 4;   // codes per group
+  constexpr int GB = GS * W;             // bits per group (<= 32)
+  constexpr int NG = N / GS;
+  constexpr uint64_t ONES = group_ones(W, GS);   // sum of 2^(W*i), i < GS
+  constexpr uint32_t KW = (uint32_t)((0x4B400000ull * ONES) & 0xffffffffull);
+#pragma unroll
+  for (int j = 0; j < N * W / 32; ++j) w[j] = 0;
+#pragma unroll
+  for (int j = 0; j < NG; ++j) {
+    uint32_t acc = __float_as_uint(t(j * GS + GS - 1));
+#pragma unroll
+    for (int i = GS - 2; i >= 0; --i) acc = acc * (1u << W) + __float_as_uint(t(j * GS + i));
+    const uint32_t g = acc - KW;
+    const int bit = j * GB, wi = bit >> 5, sh = bit & 31;
+    w[wi] |= g << sh;
+    if (sh + GB > 32) w[wi + 1] |= g >> (32 - sh);
+  }
+}
+
+// Bit stream -> dequantised values z + q*s (one fused multiply-add per code).  A code is turned into
+// a float without being shifted down: its bits, masked in place at bit p of a word (or of the word's
+// upper half), are OR-ed into the mantissa of 2^23, giving 2^23 + q*2^p exactly; subtracting 2^23 and
+// multiplying by s*2^-p inside the fused multiply-add gives the same real product q*s, so the result
+// is bit-identical to fma((float)q, s, z).
+template <int W, int N>
+__device__ __forceinline__ void unpack_dequant(const uint32_t *w, float s, float z, float (&x)[N]) {
+  constexpr uint32_t M = (1u << W) - 1u;
+#pragma unroll
+  for (int k = 0; k < N; ++k) {
+    const int bit = k * W, j = bit >> 5, sh = bit & 31;
+    uint32_t src;
+    int p;
+    if (sh + W <= 23) { src = w[j]; p = sh; }
+    else if (sh + W <= 32) { src = w[j] >> 16; p = sh - 16; }
+    else { src = __funnelshift_r(w[j], w[j + 1], sh); p = 0; }
+    const float f = __uint_as_float((src & (M << p)) | 0x4B000000u) - 8388608.0f;
+    x[k] = __fmaf_rn(f, s * (1.0f / (float)(1u << p)), z);
   }
 }
 

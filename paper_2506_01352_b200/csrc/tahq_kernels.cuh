@@ -1,14 +1,12 @@
 // Kernels of the TAH-Quant boundary codec (sm_100a).  See tahq_device.cuh for the work decomposition.
 //
-//   encode:  stats_kernel        Eq. 1-2   tile -> entropy score                 (skipped for integer budgets)
-//            hist_kernel         Sec. 3.2  per-group histogram of binned scores
-//            gather_kernel       Sec. 3.2  threshold bin + candidates of that bin
-//            resolve_kernel      Sec. 3.2  exact k_hi-th largest (score, index) key per group
-//            bitmap_kernel       Sec. 3.2  1-bit map + hi-tile counts per 128 tiles
-//            scan_kernel         Sec. 3.4  exclusive prefix of those counts (payload offsets)
-//            quant_pack_kernel   Eq. 3-4, Sec. 3.3-3.4  pivot test, swap + Hadamard, quantise, pack
-//   decode:  count_kernel + scan_kernel    bit map -> payload offsets, header check
-//            decode_kernel       Sec. 3.3, Alg. 1 l.5  unpack, z + q*s, inverse transform, store
+//   encode:  stats_kernel        Eq. 1-2   tile -> entropy score, per-group histogram of binned scores
+//                                          (skipped for integer budgets)
+//            select_kernel       Sec. 3.2  threshold bin, its candidates, exact k_hi-th (score, index) key
+//            quant_pack_kernel   Eq. 3-4, Sec. 3.2-3.4  bit map + offsets (prefix over CTAs), pivot test,
+//                                          swap + Hadamard, quantise, pack
+//   decode:  decode_kernel       Sec. 3.3, Alg. 1 l.5  header check, offsets from the bit map, unpack,
+//                                          z + q*s, inverse transform, store
 #pragma once
 
 #include "tahq_device.cuh"
@@ -24,40 +22,52 @@ struct Args {
   uint64_t off_bitmap, off_sz, off_pivot, off_payload, payload_bytes, total_bytes;
   float tau, eps_l1, eps_log, eps_ratio;
   float *scores;            // [n_tiles]
-  uint32_t *hist;           // [n_groups][kBins]
-  uint32_t *ncand;          // [n_groups]
-  uint2 *binsel;            // [n_groups] {threshold bin, rank inside the bin (1-based)}
-  unsigned long long *theta;// [n_groups] key of the k_hi-th ranked tile
+  uint32_t *hist;           // [n_groups][kBins]   (zeroed per call)
+  uint32_t *ncand;          // [n_groups]          (zeroed per call)
+  uint32_t *done;           // [n_groups]          (zeroed per call) CTAs of select_kernel that finished a group
+  unsigned long long *theta;// [n_groups] ranking key of the k_hi-th ranked tile
   unsigned long long *cand; // [n_groups][cand_cap]
-  uint32_t cand_cap, cpg;   // candidate capacity per group; CTAs per group of hist/gather
-  uint32_t direct;          // small groups: resolve_kernel ranks all scores of the group itself
-  uint32_t *cnt128;         // [ceil(n_tiles/128)+2] hi tiles per 128 tiles, then their exclusive prefix
+  uint32_t cand_cap, cpg;   // candidate capacity per group; CTAs per group of select_kernel
+  uint32_t direct;          // small groups: select_kernel ranks all scores of the group itself
+  unsigned long long *flags;// [kMaxGrid] (zeroed per call) per-CTA published counts for the offset prefix
   uint32_t *status;         // device status word
   uint32_t header[32];      // the 128-byte header of the packed buffer
 };
 
+constexpr int kMaxGrid = 2048;                               // upper bound on CTAs of the persistent tile kernels
+constexpr unsigned long long kPublished = 1ull << 63;        // flag word: count is valid
+constexpr unsigned long long kAbort = 1ull << 62;            // flag word: decode refused the buffer
+constexpr unsigned long long kCountMask = (1ull << 48) - 1;
+constexpr uint32_t kSpinLimit = 1u << 22;                    // bounded wait on a predecessor's flag
+
+// Contiguous chunk range of this CTA.
+__device__ __forceinline__ void cta_chunk_range(uint64_t n_chunks, uint64_t &c0, uint64_t &c1) {
+  c0 = n_chunks * blockIdx.x / gridDim.x;
+  c1 = n_chunks * (blockIdx.x + 1ull) / gridDim.x;
+}
+
 // ------------------------------------------------------------------------------------------
-// Persistent multi-stage cp.async loop over the chunks of a CTA
+// Persistent multi-stage cp.async loop over the chunks [c0, c1) of a CTA
 // ------------------------------------------------------------------------------------------
 template <class C, int NST, class Body>
-__device__ __forceinline__ void chunk_pipeline(const uint8_t *in, uint64_t n_tiles, uint8_t *stages, Body &&body) {
-  const uint64_t n_chunks = (n_tiles + C::TPC - 1) / C::TPC;
-  uint64_t c_issue = blockIdx.x;
+__device__ __forceinline__ void chunk_pipeline(const uint8_t *in, uint64_t n_tiles, uint64_t c0, uint64_t c1,
+                                               uint8_t *stages, Body &&body) {
+  uint64_t c_issue = c0;
 #pragma unroll
   for (int s = 0; s < NST - 1; ++s) {
-    if (c_issue < n_chunks) issue_chunk<C>(in, n_tiles, c_issue, stages + (size_t)s * C::STAGE_BYTES);
+    if (c_issue < c1) issue_chunk<C>(in, n_tiles, c_issue, stages + (size_t)s * C::STAGE_BYTES);
     cp_async_commit();
-    c_issue += gridDim.x;
+    ++c_issue;
   }
   int stage = 0;
-  for (uint64_t c = blockIdx.x; c < n_chunks; c += gridDim.x) {
+  for (uint64_t c = c0; c < c1; ++c) {
     cp_async_wait<NST - 2>();
     __syncthreads();   // chunk c has landed; everyone is done with the stage consumed last time
     {
       const int s2 = (stage + NST - 1) % NST;
-      if (c_issue < n_chunks) issue_chunk<C>(in, n_tiles, c_issue, stages + (size_t)s2 * C::STAGE_BYTES);
+      if (c_issue < c1) issue_chunk<C>(in, n_tiles, c_issue, stages + (size_t)s2 * C::STAGE_BYTES);
       cp_async_commit();
-      c_issue += gridDim.x;
+      ++c_issue;
     }
     body(c, stages + (size_t)stage * C::STAGE_BYTES);
     stage = (stage + 1) % NST;
@@ -65,107 +75,127 @@ __device__ __forceinline__ void chunk_pipeline(const uint8_t *in, uint64_t n_til
   cp_async_wait<0>();
 }
 
+// Exclusive prefix over the CTAs of the grid of one count per CTA (hi tiles in the CTA's range), which
+// fixes where the CTA's payload starts (Sec. 3.4).  CTAs publish their count in a zeroed flag array
+// and read every predecessor's; lower CTAs are dispatched first, so a waiting CTA only ever waits for
+// CTAs that are running.  Every wait is bounded: on expiry the status word gets TAHQ_DEV_TIMEOUT.
+__device__ __forceinline__ uint64_t cta_exclusive_prefix(const Args &a, uint64_t mine, bool abort_in, bool &abort_out) {
+  __shared__ unsigned long long s_sum[kThreads / 32];
+  __shared__ uint32_t s_abort;
+  if (threadIdx.x == 0) {
+    s_abort = 0;
+    __threadfence();
+    atomicExch(a.flags + blockIdx.x, kPublished | (abort_in ? kAbort : 0ull) | (mine & kCountMask));
+  }
+  __syncthreads();
+  unsigned long long sum = 0;
+  bool ab = false;
+  for (uint32_t j = threadIdx.x; j < blockIdx.x; j += kThreads) {
+    const volatile unsigned long long *f = a.flags + j;
+    unsigned long long v = *f;
+    uint32_t spins = 0;
+    while (!(v & kPublished) && ++spins < kSpinLimit) v = *f;
+    if (!(v & kPublished)) { atomicOr(a.status, 4u /* TAHQ_DEV_TIMEOUT */); v = 0; }
+    sum += v & kCountMask;
+    ab |= (v & kAbort) != 0;
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(kFull, sum, o);
+  if ((threadIdx.x & 31) == 0) s_sum[threadIdx.x >> 5] = sum;
+  if (ab) s_abort = 1;
+  __syncthreads();
+  unsigned long long total = 0;
+#pragma unroll
+  for (int w = 0; w < kThreads / 32; ++w) total += s_sum[w];
+  abort_out = abort_in || s_abort != 0;
+  __syncthreads();
+  return total;
+}
+
 // ------------------------------------------------------------------------------------------
-// Eq. 1-2: entropy score per tile
+// Eq. 1-2: entropy score per tile, plus the per-group histogram of binned scores (Sec. 3.2)
 // ------------------------------------------------------------------------------------------
 template <class C, int NST>
 __global__ void __launch_bounds__(kThreads) stats_kernel(const Args a) {
   extern __shared__ __align__(128) uint8_t smem[];
-  chunk_pipeline<C, NST>(a.in, a.n_tiles, smem, [&](uint64_t c, const uint8_t *stage) {
+  __shared__ uint32_t s_hist[kBins];
+  const bool use_hist = !a.direct;
+  if (use_hist) {
+    for (int b = threadIdx.x; b < kBins; b += kThreads) s_hist[b] = 0;
+    __syncthreads();
+  }
+  auto flush = [&](uint64_t g) {   // add this CTA's counts of group g to the global histogram
+    __syncthreads();
+    uint32_t *gh = a.hist + g * kBins;
+    for (int b = threadIdx.x; b < kBins; b += kThreads) {
+      const uint32_t v = s_hist[b];
+      if (v) { atomicAdd(gh + b, v); s_hist[b] = 0; }
+    }
+    __syncthreads();
+  };
+  const uint64_t n_chunks = (a.n_tiles + C::TPC - 1) / C::TPC;
+  uint64_t c0, c1;
+  cta_chunk_range(n_chunks, c0, c1);
+  long long gcur = -1;
+  chunk_pipeline<C, NST>(a.in, a.n_tiles, c0, c1, smem, [&](uint64_t c, const uint8_t *stage) {
     const float s = tile_score<C>(stage, a.eps_l1, a.eps_log);
-    const uint64_t tile = c * C::TPC + threadIdx.x / C::LPT;
-    if (tile < a.n_tiles && (C::LPT == 1 || !(threadIdx.x & 1))) a.scores[tile] = s;
+    const uint64_t tile0 = c * C::TPC;
+    const uint64_t tile = tile0 + threadIdx.x / C::LPT;
+    const bool mine = tile < a.n_tiles && (C::LPT == 1 || !(threadIdx.x & 1));
+    if (mine) a.scores[tile] = s;
+    if (use_hist) {
+      const uint64_t last = (tile0 + C::TPC <= a.n_tiles ? tile0 + C::TPC : a.n_tiles) - 1;
+      const uint64_t g0 = tile0 / a.tiles_per_group, g1 = last / a.tiles_per_group;
+      if (g0 == g1) {
+        if ((long long)g0 != gcur) {
+          if (gcur >= 0) flush((uint64_t)gcur);
+          gcur = (long long)g0;
+        }
+        if (mine) atomicAdd(&s_hist[score_bin(s)], 1u);
+      } else if (mine) {   // a chunk that straddles two ranking groups goes straight to global memory
+        atomicAdd(a.hist + (tile / a.tiles_per_group) * kBins + score_bin(s), 1u);
+      }
+    }
   });
+  if (use_hist && gcur >= 0) flush((uint64_t)gcur);
 }
 
 // ------------------------------------------------------------------------------------------
-// Sec. 3.2: exact top-k_hi per ranking group
+// Sec. 3.2: exact top-k_hi per ranking group -> theta[g], the ranking key of the k_hi-th tile
 // ------------------------------------------------------------------------------------------
-__device__ __forceinline__ void group_slice(const Args &a, uint64_t &g, uint64_t &lo, uint64_t &hi) {
-  g = blockIdx.x / a.cpg;
-  const uint64_t j = blockIdx.x % a.cpg;
-  const uint64_t slice = (a.tiles_per_group + a.cpg - 1) / a.cpg;
-  lo = j * slice;
-  hi = lo + slice < a.tiles_per_group ? lo + slice : a.tiles_per_group;
-  if (lo > hi) lo = hi;
-}
+constexpr int kSelThreads = 1024;
+constexpr int kSortCap = 8192;   // candidates that are sorted in shared memory
 
-__global__ void __launch_bounds__(kThreads) hist_kernel(const Args a) {
-  __shared__ uint32_t h[kBins];
-  for (int b = threadIdx.x; b < kBins; b += kThreads) h[b] = 0;
-  __syncthreads();
-  uint64_t g, lo, hi;
-  group_slice(a, g, lo, hi);
-  const float *sc = a.scores + g * a.tiles_per_group;
-  for (uint64_t i = lo + threadIdx.x; i < hi; i += kThreads) atomicAdd(&h[score_bin(sc[i])], 1u);
-  __syncthreads();
-  uint32_t *gh = a.hist + g * kBins;
-  for (int b = threadIdx.x; b < kBins; b += kThreads)
-    if (h[b]) atomicAdd(&gh[b], h[b]);
-}
-
-__global__ void __launch_bounds__(kThreads) gather_kernel(const Args a) {
-  __shared__ uint32_t h[kBins];
-  __shared__ uint32_t part[kThreads];
-  __shared__ uint32_t sel[2];
-  uint64_t g, lo, hi;
-  group_slice(a, g, lo, hi);
-  const uint32_t *gh = a.hist + g * kBins;
-  for (int b = threadIdx.x; b < kBins; b += kThreads) h[b] = gh[b];
-  __syncthreads();
-  constexpr int BPT = kBins / kThreads;   // bins per thread
-  uint32_t mine = 0;
-#pragma unroll
-  for (int j = 0; j < BPT; ++j) mine += h[threadIdx.x * BPT + j];
-  part[threadIdx.x] = mine;
-  __syncthreads();
-  uint32_t above = 0;   // tiles in bins above this thread's range
-  for (int j = threadIdx.x + 1; j < kThreads; ++j) above += part[j];
-  const uint32_t k = (uint32_t)a.k_hi;
-  if (above < k && above + mine >= k) {   // the k-th ranked tile lies in one of this thread's bins
-    for (int j = BPT - 1; j >= 0; --j) {
-      const uint32_t n = h[threadIdx.x * BPT + j];
-      if (above + n >= k) { sel[0] = threadIdx.x * BPT + j; sel[1] = k - above; break; }
-      above += n;
-    }
-  }
-  __syncthreads();
-  const uint32_t B = sel[0];
-  if (blockIdx.x % a.cpg == 0 && threadIdx.x == 0) a.binsel[g] = make_uint2(B, sel[1]);
-  const float *sc = a.scores + g * a.tiles_per_group;
-  for (uint64_t i = lo + threadIdx.x; i < hi; i += kThreads) {
-    const float s = sc[i];
-    if (score_bin(s) == B) {
-      const uint32_t slot = atomicAdd(&a.ncand[g], 1u);
-      if (slot < a.cand_cap) a.cand[g * a.cand_cap + slot] = rank_key(s, (uint32_t)i);
+// Bitonic sort, descending, of n = 2^m keys in shared memory by the whole CTA.
+__device__ __forceinline__ void bitonic_desc(unsigned long long *s, uint32_t n) {
+  for (uint32_t k = 2; k <= n; k <<= 1) {
+    for (uint32_t j = k >> 1; j > 0; j >>= 1) {
+      for (uint32_t i = threadIdx.x; i < n; i += kSelThreads) {
+        const uint32_t p = i ^ j;
+        if (p > i) {
+          const unsigned long long x = s[i], y = s[p];
+          const bool desc = (i & k) == 0;
+          if (desc ? (x < y) : (x > y)) { s[i] = y; s[p] = x; }
+        }
+      }
+      __syncthreads();
     }
   }
 }
 
-constexpr int kResolveThreads = 1024;
-
-// r-th largest 64-bit key among the candidates of the threshold bin: radix select, 8 bits a pass.
-__global__ void __launch_bounds__(kResolveThreads) resolve_kernel(const Args a) {
+// r-th largest (1-based) key of a sequence, radix select with 8 bits a pass.  get(i, key) returns
+// false for entries that do not take part.
+template <class Get>
+__device__ __forceinline__ unsigned long long radix_select(uint64_t count, uint32_t r, Get &&get) {
   __shared__ uint32_t h[256];
   __shared__ uint32_t pick[2];
-  const uint64_t g = blockIdx.x;
-  const uint32_t B = a.direct ? 0u : a.binsel[g].x;
-  uint32_t r = a.direct ? (uint32_t)a.k_hi : a.binsel[g].y;
-  const uint32_t n = a.direct ? 0u : a.hist[g * kBins + B];
-  const bool listed = !a.direct && n <= a.cand_cap;   // otherwise take the candidates from the scores
-  const unsigned long long *cand = a.cand + g * a.cand_cap;
-  const float *sc = a.scores + g * a.tiles_per_group;
-  const uint64_t count = listed ? n : a.tiles_per_group;
   unsigned long long prefix = 0, mask = 0;
   for (int shift = 56; shift >= 0; shift -= 8) {
     if (threadIdx.x < 256) h[threadIdx.x] = 0;
     __syncthreads();
-    for (uint64_t i = threadIdx.x; i < count; i += kResolveThreads) {
+    for (uint64_t i = threadIdx.x; i < count; i += kSelThreads) {
       unsigned long long key;
-      bool ok;
-      if (listed) { key = cand[i]; ok = true; }
-      else { const float s = sc[i]; ok = a.direct || score_bin(s) == B; key = rank_key(s, (uint32_t)i); }
-      if (ok && (key & mask) == prefix) atomicAdd(&h[(unsigned)(key >> shift) & 255u], 1u);
+      if (get(i, key) && (key & mask) == prefix) atomicAdd(&h[(unsigned)(key >> shift) & 255u], 1u);
     }
     __syncthreads();
     if (threadIdx.x < 32) {
@@ -195,135 +225,349 @@ __global__ void __launch_bounds__(kResolveThreads) resolve_kernel(const Args a) 
     r = pick[1];
     __syncthreads();
   }
-  if (threadIdx.x == 0) a.theta[g] = prefix;
+  return prefix;
 }
 
-// Bit map (tile t -> bit t&31 of word t>>5) and the number of hi tiles in every 128 tiles.
-__global__ void __launch_bounds__(kThreads) bitmap_kernel(const Args a) {
-  __shared__ uint32_t wc[kThreads / 32];
-  const uint64_t t = (uint64_t)blockIdx.x * kThreads + threadIdx.x;
-  bool hi = false;
-  if (t < a.n_tiles) {
-    const uint64_t g = t / a.tiles_per_group;
-    const uint32_t i = (uint32_t)(t - g * a.tiles_per_group);
-    hi = rank_key(a.scores[t], i) >= a.theta[g];
-  }
-  const uint32_t word = __ballot_sync(kFull, hi);
+__global__ void __launch_bounds__(kSelThreads) select_kernel(const Args a) {
+  extern __shared__ __align__(16) unsigned long long s_keys[];   // kSortCap keys
+  __shared__ uint32_t s_warp[kSelThreads / 32];
+  __shared__ uint32_t s_sel[2];
+  __shared__ uint32_t s_last;
+  const uint64_t g = blockIdx.x / a.cpg;
+  const uint64_t ng = a.tiles_per_group;
+  const float *sc = a.scores + g * ng;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  if (lane == 0) {
-    reinterpret_cast<uint32_t *>(a.packed + a.off_bitmap)[t >> 5] = word;
-    wc[warp] = __popc(word);
-  }
-  __syncthreads();
-  if (threadIdx.x < 2)
-    a.cnt128[(uint64_t)blockIdx.x * 2 + threadIdx.x] =
-        wc[4 * threadIdx.x] + wc[4 * threadIdx.x + 1] + wc[4 * threadIdx.x + 2] + wc[4 * threadIdx.x + 3];
-}
 
-// Single-CTA exclusive scan of cnt128[0..n) in place.  expect_total != ~0: flag a mismatch.
-constexpr int kScanThreads = 1024;
-__global__ void __launch_bounds__(kScanThreads) scan_kernel(uint32_t *v, uint64_t n, unsigned long long expect_total,
-                                                            uint32_t *status) {
-  __shared__ uint32_t wsum[32];
-  const uint64_t per = (n + kScanThreads - 1) / kScanThreads;
-  const uint64_t lo = per * threadIdx.x;
-  const uint64_t hi = lo + per < n ? lo + per : n;
-  uint32_t mine = 0;
-  for (uint64_t i = lo; i < hi; ++i) mine += v[i];
+  auto sort_and_pick = [&](uint32_t n, uint32_t r) {   // keys [0, n) are in s_keys
+    uint32_t n2 = 2;
+    while (n2 < n) n2 <<= 1;
+    for (uint32_t i = n + threadIdx.x; i < n2; i += kSelThreads) s_keys[i] = 0;   // below every real key
+    __syncthreads();
+    bitonic_desc(s_keys, n2);
+    if (threadIdx.x == 0) a.theta[g] = s_keys[r - 1];
+  };
+
+  if (a.direct) {   // small group: rank all of its tiles here (one CTA per group)
+    for (uint32_t i = threadIdx.x; i < (uint32_t)ng; i += kSelThreads) s_keys[i] = rank_key(sc[i], i);
+    __syncthreads();
+    sort_and_pick((uint32_t)ng, (uint32_t)a.k_hi);
+    return;
+  }
+
+  // ---- A: the bin that holds the k_hi-th ranked tile (every CTA of the group finds it for itself)
+  const uint32_t *gh = a.hist + g * kBins;
+  constexpr int BPT = kBins / kSelThreads;
+  uint32_t hb[BPT], mine = 0;
+#pragma unroll
+  for (int j = 0; j < BPT; ++j) { hb[j] = gh[threadIdx.x * BPT + j]; mine += hb[j]; }
+  // suffix sums: tiles in bins above this thread's bins
   uint32_t incl = mine;
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 #pragma unroll
   for (int o = 1; o < 32; o *= 2) {
-    const uint32_t u = __shfl_up_sync(kFull, incl, o);
-    if (lane >= o) incl += u;
+    const uint32_t v = __shfl_down_sync(kFull, incl, o);
+    if (lane + o < 32) incl += v;
   }
-  if (lane == 31) wsum[warp] = incl;
+  if (lane == 0) s_warp[warp] = incl;
   __syncthreads();
-  if (warp == 0) {
-    const uint32_t w = wsum[lane];
-    uint32_t wi = w;
+  uint32_t above = incl - mine;
+  for (int w = warp + 1; w < kSelThreads / 32; ++w) above += s_warp[w];
+  const uint32_t k = (uint32_t)a.k_hi;
+  if (above < k && above + mine >= k) {
 #pragma unroll
-    for (int o = 1; o < 32; o *= 2) {
-      const uint32_t u = __shfl_up_sync(kFull, wi, o);
-      if (lane >= o) wi += u;
+    for (int j = BPT - 1; j >= 0; --j) {
+      if (above < k && above + hb[j] >= k) { s_sel[0] = threadIdx.x * BPT + j; s_sel[1] = k - above; }
+      above += hb[j];
     }
-    wsum[lane] = wi - w;
-    if (lane == 31 && expect_total != ~0ull && (unsigned long long)wi != expect_total)
-      atomicOr(status, 2u /* TAHQ_DEV_BAD_BITMAP */);
   }
   __syncthreads();
-  uint32_t run = wsum[warp] + incl - mine;
-  for (uint64_t i = lo; i < hi; ++i) {
-    const uint32_t c = v[i];
-    v[i] = run;
-    run += c;
+  const uint32_t B = s_sel[0], r = s_sel[1];
+
+  // ---- B: this CTA's slice of the group: candidates of bin B go to the group's list
+  const uint64_t j = blockIdx.x % a.cpg;
+  const uint64_t slice = (ng + a.cpg - 1) / a.cpg;
+  const uint64_t lo = j * slice < ng ? j * slice : ng;
+  const uint64_t hi = lo + slice < ng ? lo + slice : ng;
+  for (uint64_t i0 = lo; i0 < hi; i0 += kSelThreads) {   // whole warps stay in the loop: one atomic per warp
+    const uint64_t i = i0 + threadIdx.x;
+    const float s = i < hi ? sc[i] : 0.0f;
+    const bool take = i < hi && score_bin(s) == B;
+    const unsigned m = __ballot_sync(kFull, take);
+    if (m) {
+      uint32_t base = 0;
+      if (lane == 0) base = atomicAdd(&a.ncand[g], (uint32_t)__popc(m));
+      base = __shfl_sync(kFull, base, 0);
+      const uint32_t slot = base + __popc(m & ((1u << lane) - 1u));
+      if (take && slot < a.cand_cap) a.cand[g * a.cand_cap + slot] = rank_key(s, (uint32_t)i);
+    }
+  }
+
+  // ---- C: the CTA that finishes the group last ranks the candidates exactly
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) s_last = atomicAdd(&a.done[g], 1u) == a.cpg - 1;
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  const uint32_t n = gh[B];
+  const unsigned long long *cand = a.cand + g * a.cand_cap;
+  if (n <= a.cand_cap && n <= (uint32_t)kSortCap) {
+    for (uint32_t i = threadIdx.x; i < n; i += kSelThreads) s_keys[i] = __ldcg(cand + i);
+    __syncthreads();
+    sort_and_pick(n, r);
+  } else if (n <= a.cand_cap) {
+    const unsigned long long t = radix_select(n, r, [&](uint64_t i, unsigned long long &key) {
+      key = __ldcg(cand + i);
+      return true;
+    });
+    if (threadIdx.x == 0) a.theta[g] = t;
+  } else {   // more candidates than the list holds: take them from the scores
+    const unsigned long long t = radix_select(ng, r, [&](uint64_t i, unsigned long long &key) {
+      const float s = sc[i];
+      key = rank_key(s, (uint32_t)i);
+      return score_bin(s) == B;
+    });
+    if (threadIdx.x == 0) a.theta[g] = t;
   }
 }
 
+// Is tile `tile` one of the k_hi highest-ranked tiles of its group?
+__device__ __forceinline__ bool tile_is_hi(const Args &a, uint64_t tile) {
+  const uint64_t g = tile / a.tiles_per_group;
+  const uint32_t i = (uint32_t)(tile - g * a.tiles_per_group);
+  return rank_key(__ldg(a.scores + tile), i) >= a.theta[g];
+}
+
 // ------------------------------------------------------------------------------------------
-// Widths and offsets of the tiles of one chunk, from the chunk's words of the bit map
+// Widths and offsets inside one chunk of kThreads rows
 // ------------------------------------------------------------------------------------------
-template <class C>
-struct ChunkPlan {
-  uint32_t is_hi;       // this thread's tile uses the higher width
-  uint32_t row_off;     // byte offset of this thread's codes inside the chunk's payload
-  uint32_t bytes;       // payload bytes of the chunk
-  uint64_t goff;        // byte offset of the chunk's payload inside the payload section
+
+// Position of a tile inside its ranking group, kept incrementally while a CTA walks consecutive tiles.
+struct GroupCursor {
+  uint64_t g;     // ranking group of the chunk's first tile
+  uint32_t rem;   // index of that tile inside the group
+  __device__ __forceinline__ void init(const Args &a, uint64_t tile0) {
+    g = tile0 / a.tiles_per_group;
+    rem = (uint32_t)(tile0 - g * a.tiles_per_group);
+  }
+  __device__ __forceinline__ void advance(const Args &a, uint32_t n) {
+    uint64_t r = (uint64_t)rem + n;
+    if (r >= a.tiles_per_group) { g += r / a.tiles_per_group; r %= a.tiles_per_group; }
+    rem = (uint32_t)r;
+  }
+  // is the tile `off` tiles after the cursor among the k_hi highest-ranked of its group?
+  __device__ __forceinline__ bool is_hi(const Args &a, uint64_t tile, uint32_t off) const {
+    uint64_t gg = g;
+    uint64_t i = (uint64_t)rem + off;
+    if (i >= a.tiles_per_group) { gg += i / a.tiles_per_group; i %= a.tiles_per_group; }
+    return rank_key(__ldg(a.scores + tile), (uint32_t)i) >= __ldg(a.theta + gg);
+  }
 };
 
-template <class C>
-__device__ __forceinline__ ChunkPlan<C> plan_chunk(const Args &a, uint64_t c) {
-  constexpr int NW = C::TPC / 32;
-  const uint64_t tile0 = c * C::TPC;
-  const int r = threadIdx.x / C::LPT, half = threadIdx.x % C::LPT;
-  const int myw = r >> 5, mybit = r & 31;
-  uint32_t hi_before = 0, total_hi = 0, myword = 0;
-  if (a.mixed) {
-    const uint32_t *bm = reinterpret_cast<const uint32_t *>(a.packed + a.off_bitmap) + tile0 / 32;
+__device__ __forceinline__ uint32_t block_sum(uint32_t v) {
+  __shared__ uint32_t s_part[kThreads / 32];
 #pragma unroll
-    for (int w = 0; w < NW; ++w) {
-      const uint64_t first = tile0 + 32ull * w;
-      uint32_t word = 0;
-      if (first < a.n_tiles) {
-        const uint64_t left = a.n_tiles - first;
-        word = __ldg(bm + w) & (left >= 32 ? 0xffffffffu : ((1u << (uint32_t)left) - 1u));
-      }
-      const uint32_t pc = __popc(word);
-      total_hi += pc;
-      hi_before += (w < myw) ? pc : 0u;
-      myword = (w == myw) ? word : myword;
-    }
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(kFull, v, o);
+  if ((threadIdx.x & 31) == 0) s_part[threadIdx.x >> 5] = v;
+  __syncthreads();
+  uint32_t t = 0;
+#pragma unroll
+  for (int w = 0; w < kThreads / 32; ++w) t += s_part[w];
+  __syncthreads();
+  return t;
+}
+
+// One-lane-per-tile kernels: stable counting sort of the CTA's 256 tiles by class
+// (bit 0 = higher width, bit 1 = transformed) so that warps become uniform, fused with the running
+// count of higher-width tiles that fixes every tile's payload offset.  `mid` runs between the two
+// barriers (after hi_before / total_hi are known, before the permutation is read).
+struct Regroup {
+  int src, cls;
+  uint32_t hi_before, total_hi, hi_ballot;
+};
+template <class Mid>
+__device__ __forceinline__ Regroup regroup(int cls, uint8_t *s_perm, uint2 *s_cnt, Mid &&mid) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const unsigned b1 = __ballot_sync(kFull, cls & 1), b2 = __ballot_sync(kFull, cls & 2);
+  const unsigned m0 = ~b1 & ~b2, m1 = b1 & ~b2, m2 = ~b1 & b2, m3 = b1 & b2;
+  if (lane == 0) s_cnt[warp] = make_uint2(__popc(m0) | (__popc(m1) << 16), __popc(m2) | (__popc(m3) << 16));
+  __syncthreads();
+  uint32_t tot_lo = 0, tot_hi = 0, bef_lo = 0, bef_hi = 0;   // two 16-bit counters per word
+#pragma unroll
+  for (int w = 0; w < kThreads / 32; ++w) {
+    const uint2 c = s_cnt[w];
+    tot_lo += c.x; tot_hi += c.y;
+    bef_lo += (w < warp) ? c.x : 0u;
+    bef_hi += (w < warp) ? c.y : 0u;
   }
-  hi_before += __popc(myword & ((1u << mybit) - 1u));
-  ChunkPlan<C> p;
-  p.is_hi = (myword >> mybit) & 1u;
-  const uint32_t b = a.lo + p.is_hi;
-  p.row_off = (C::G / 8) * (a.lo * r + hi_before) + half * (C::EPT / 8) * b;
-  const uint64_t left = a.n_tiles - tile0;
-  const uint32_t nvalid = left < (uint64_t)C::TPC ? (uint32_t)left : (uint32_t)C::TPC;
-  p.bytes = (C::G / 8) * (a.lo * nvalid + total_hi);
-  const uint64_t P = a.mixed ? (uint64_t)__ldg(a.cnt128 + tile0 / 128) : 0ull;
-  p.goff = (uint64_t)(C::G / 8) * ((uint64_t)a.lo * tile0 + P);
-  return p;
+  const int base1 = tot_lo & 0xffff, base2 = base1 + (tot_lo >> 16), base3 = base2 + (tot_hi & 0xffff);
+  const unsigned mine = (cls == 0) ? m0 : (cls == 1) ? m1 : (cls == 2) ? m2 : m3;
+  const int before = (cls == 0) ? (bef_lo & 0xffff) : (cls == 1) ? (bef_lo >> 16) : (cls == 2) ? (bef_hi & 0xffff)
+                                                                                               : (bef_hi >> 16);
+  const int base = (cls == 0) ? 0 : (cls == 1) ? base1 : (cls == 2) ? base2 : base3;
+  const unsigned lt = (1u << lane) - 1u;
+  Regroup r;
+  r.hi_before = (bef_lo >> 16) + (bef_hi >> 16) + __popc(b1 & lt);
+  r.total_hi = (tot_lo >> 16) + (tot_hi >> 16);
+  r.hi_ballot = b1;
+  mid(r);
+  s_perm[base + before + __popc(mine & lt)] = (uint8_t)threadIdx.x;
+  __syncthreads();
+  r.src = s_perm[threadIdx.x];
+  const int t = threadIdx.x;
+  r.cls = (t >= base1) + (t >= base2) + (t >= base3);
+  return r;
+}
+
+// Two-lanes-per-tile kernels (128-wide tiles): only the running count, no regrouping.
+__device__ __forceinline__ void pair_scan(bool hi, uint32_t *s_cnt32, uint32_t &hi_before, uint32_t &total_hi,
+                                          uint32_t &tiles16) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const unsigned b = __ballot_sync(kFull, hi) & 0x55555555u;   // one bit per tile (its even lane)
+  if (lane == 0) s_cnt32[warp] = __popc(b);
+  __syncthreads();
+  uint32_t tot = 0, bef = 0;
+#pragma unroll
+  for (int w = 0; w < kThreads / 32; ++w) {
+    const uint32_t c = s_cnt32[w];
+    tot += c;
+    bef += (w < warp) ? c : 0u;
+  }
+  hi_before = bef + __popc(b & ((1u << (lane & ~1)) - 1u));
+  total_hi = tot;
+  uint32_t x = b;   // gather the even bits into the low 16: the warp's 16 tiles as they sit in the bit map
+  x = (x | (x >> 1)) & 0x33333333u;
+  x = (x | (x >> 2)) & 0x0f0f0f0fu;
+  x = (x | (x >> 4)) & 0x00ff00ffu;
+  x = (x | (x >> 8)) & 0x0000ffffu;
+  tiles16 = x;
+  __syncthreads();
 }
 
 // ------------------------------------------------------------------------------------------
 // Eq. 3-4 + Sec. 3.3-3.4: pivot test, swap + Hadamard, min-max quantisation, packing
 // ------------------------------------------------------------------------------------------
-template <class C, int W>
-__device__ __forceinline__ void pack_store(const uint32_t (&code)[C::EPT], uint32_t *dst) {
-  uint32_t w[C::EPT * W / 32];
-  pack_words<W, C::EPT>(code, w);
+constexpr float kMagic = 12582912.0f;   // 1.5 * 2^23: adding it rounds to the nearest integer, ties to even
+
+template <class C>
+__device__ __forceinline__ constexpr float hadamard_scale() {
+  return (C::G == 32) ? 0.17677669529663687f : (C::G == 64) ? 0.125f : 0.08838834764831845f;
+}
+
+// Range of a row -> binary16 zero-point and scale, and the reciprocal the codes are computed with.
+struct Quantiser {
+  float z, inv_s, qmax;
+  uint32_t sz;   // {f16 scale, f16 zero} as stored
+};
+__device__ __forceinline__ Quantiser make_quantiser(float mn, float mx, uint32_t bits) {
+  Quantiser q;
+  q.qmax = (float)((1u << bits) - 1u);
+  mn = mn + 0.0f;
+  mn = fminf(fmaxf(mn, -65504.0f), 65504.0f);
+  const __half zh = __float2half_rn(mn);
+  q.z = __half2float(zh);
+  float s = __fdiv_rn(mx - q.z, q.qmax);
+  s = (s > 0.0f) ? s : 0.0f;
+  s = fminf(s, 65504.0f);
+  const __half sh = __float2half_rn(s);
+  const float sf = __half2float(sh);
+  q.inv_s = sf > 0.0f ? __frcp_rn(sf) : 0.0f;
+  q.sz = (uint32_t)__half_as_ushort(sh) | ((uint32_t)__half_as_ushort(zh) << 16);
+  return q;
+}
+
+// t[k] = clamp((x[k] - z) * inv_s, 0, qmax) + 1.5*2^23.  The clamp is skipped when the whole warp's
+// rows provably stay inside [-0.5, qmax + 0.5) (the two operations are monotone in x), where it
+// cannot change the rounded code.
+template <int N>
+__device__ __forceinline__ void quantise_row(float (&x)[N], float mn, float mx, const Quantiser &q) {
+  const float ymin = (mn - q.z) * q.inv_s, ymax = (mx - q.z) * q.inv_s;
+  const bool safe = ymin >= -0.5f && ymax < q.qmax + 0.5f;
+  if (__all_sync(__activemask(), safe)) {
 #pragma unroll
-  for (int j = 0; j < C::EPT * W / 32; ++j) dst[j] = w[j];
+    for (int k = 0; k < N; ++k) x[k] = (x[k] - q.z) * q.inv_s + kMagic;
+  } else {
+#pragma unroll
+    for (int k = 0; k < N; ++k) x[k] = fminf(fmaxf((x[k] - q.z) * q.inv_s, 0.0f), q.qmax) + kMagic;
+  }
+}
+
+// t(k) must return q_k + 1.5*2^23 for a compile-time k; the codes leave as N*bits/32 words.
+template <int N, class F>
+__device__ __forceinline__ void pack_row(F &&t, uint32_t bits, uint32_t *dst) {
+  uint32_t w[N / 4];
+  switch (bits) {
+    case 2: pack_magic<2, N>(t, w); break;
+    case 3: pack_magic<3, N>(t, w); break;
+    case 4: pack_magic<4, N>(t, w); break;
+    case 5: pack_magic<5, N>(t, w); break;
+    case 6: pack_magic<6, N>(t, w); break;
+    case 7: pack_magic<7, N>(t, w); break;
+    default: pack_magic<8, N>(t, w); break;
+  }
+  if constexpr (N == 64) {   // 64-wide rows start on 8-byte boundaries of the staging buffer
+#pragma unroll
+    for (int j = 0; j < N / 8; ++j)
+      if (j < (int)(N * bits / 64)) reinterpret_cast<uint2 *>(dst)[j] = make_uint2(w[2 * j], w[2 * j + 1]);
+  } else {
+#pragma unroll
+    for (int j = 0; j < N / 4; ++j)
+      if (j < (int)(N * bits / 32)) dst[j] = w[j];
+  }
+}
+
+// Unflagged bf16 rows never need their elements widened one by one: min/max run on the packed
+// words, and the quantiser's first operation takes the bf16 half as an operand.
+template <class C>
+__device__ __forceinline__ Quantiser encode_raw_bf16_row(const uint8_t *stage, int row, uint32_t bits, uint32_t *dst,
+                                                          bool store) {
+  uint32_t w[C::EPT / 2];
+#pragma unroll
+  for (int q = 0; q < C::CPR; ++q) {
+    const uint4 v = *reinterpret_cast<const uint4 *>(stage + (size_t)phys_chunk<C>(row, q) * 16);
+    w[4 * q] = v.x; w[4 * q + 1] = v.y; w[4 * q + 2] = v.z; w[4 * q + 3] = v.w;
+  }
+  uint32_t lo0 = w[0], lo1 = w[1], hi0 = w[0], hi1 = w[1];
+#pragma unroll
+  for (int j = 2; j < C::EPT / 2; j += 2) {
+    lo0 = bf2_min(lo0, w[j]); hi0 = bf2_max(hi0, w[j]);
+    lo1 = bf2_min(lo1, w[j + 1]); hi1 = bf2_max(hi1, w[j + 1]);
+  }
+  lo0 = bf2_min(lo0, lo1); hi0 = bf2_max(hi0, hi1);
+  const float mn = fminf(__uint_as_float(lo0 << 16), __uint_as_float(lo0 & 0xffff0000u));
+  const float mx = fmaxf(__uint_as_float(hi0 << 16), __uint_as_float(hi0 & 0xffff0000u));
+  const Quantiser q = make_quantiser(mn, mx, bits);
+  const float ymin = (mn - q.z) * q.inv_s, ymax = (mx - q.z) * q.inv_s;
+  const bool safe = ymin >= -0.5f && ymax < q.qmax + 0.5f;
+  const float nz = -q.z;   // x + (-z) is x - z
+  if (__all_sync(__activemask(), safe)) {
+    auto t = [&](int k) {
+      float a, b;
+      bf2_add_f32(w[k >> 1], nz, a, b);
+      return ((k & 1) ? b : a) * q.inv_s + kMagic;
+    };
+    if (store) pack_row<C::EPT>(t, bits, dst);
+  } else {
+    auto t = [&](int k) {
+      float a, b;
+      bf2_add_f32(w[k >> 1], nz, a, b);
+      return fminf(fmaxf(((k & 1) ? b : a) * q.inv_s, 0.0f), q.qmax) + kMagic;
+    };
+    if (store) pack_row<C::EPT>(t, bits, dst);
+  }
+  return q;
 }
 
 template <class C, int NST>
-__global__ void __launch_bounds__(kThreads) quant_pack_kernel(const Args a) {
+__global__ void __launch_bounds__(kThreads, 2) quant_pack_kernel(const Args a) {
   extern __shared__ __align__(128) uint8_t smem[];
   uint32_t *out = reinterpret_cast<uint32_t *>(smem + (size_t)NST * C::STAGE_BYTES);
+  __shared__ uint8_t s_perm[kThreads];
+  __shared__ uint2 s_cnt[kThreads / 32];
+  __shared__ uint16_t s_rowoff[kThreads];
+  __shared__ float s_a1[kThreads];
   uint32_t *sz32 = reinterpret_cast<uint32_t *>(a.packed + a.off_sz);
   uint8_t *pivot = a.packed + a.off_pivot;
+  uint32_t *bitmap = reinterpret_cast<uint32_t *>(a.packed + a.off_bitmap);
 
   if (blockIdx.x == 0) {   // header and the zero padding behind every section
     if (threadIdx.x < 32) reinterpret_cast<uint32_t *>(a.packed)[threadIdx.x] = a.header[threadIdx.x];
@@ -335,62 +579,141 @@ __global__ void __launch_bounds__(kThreads) quant_pack_kernel(const Args a) {
       for (uint64_t o = pad[s][0] + threadIdx.x; o < pad[s][1]; o += kThreads) a.packed[o] = 0;
   }
 
-  chunk_pipeline<C, NST>(a.in, a.n_tiles, smem, [&](uint64_t c, const uint8_t *stage) {
+  const uint64_t n_chunks = (a.n_tiles + C::TPC - 1) / C::TPC;
+  uint64_t c0, c1;
+  cta_chunk_range(n_chunks, c0, c1);
+  GroupCursor cur;
+  cur.init(a, c0 * C::TPC);
+
+  // Sec. 3.4: where this CTA's payload starts = higher-width tiles of all CTAs before it
+  uint64_t hi_run = 0;
+  if (a.mixed) {
+    const uint64_t t0 = c0 * C::TPC, t1 = c1 * C::TPC < a.n_tiles ? c1 * C::TPC : a.n_tiles;
+    GroupCursor pc = cur;
+    uint32_t n = 0;
+    for (uint64_t tb = t0; tb < t1; tb += kThreads) {
+      const uint64_t t = tb + threadIdx.x;
+      if (t < t1) n += pc.is_hi(a, t, threadIdx.x) ? 1u : 0u;
+      pc.advance(a, kThreads);
+    }
+    bool unused;
+    hi_run = cta_exclusive_prefix(a, block_sum(n), false, unused);
+  }
+
+  chunk_pipeline<C, NST>(a.in, a.n_tiles, c0, c1, smem, [&](uint64_t c, const uint8_t *stage) {
     const uint64_t tile0 = c * C::TPC;
-    const int half = threadIdx.x % C::LPT;
-    const uint64_t tile = tile0 + threadIdx.x / C::LPT;
-    const bool valid = tile < a.n_tiles;
-    const ChunkPlan<C> plan = plan_chunk<C>(a, c);
-    if (!a.mixed && threadIdx.x < C::TPC / 32)   // integer budget: the bit map is all zero
-      reinterpret_cast<uint32_t *>(a.packed + a.off_bitmap)[tile0 / 32 + threadIdx.x] = 0;
+    const uint64_t left = a.n_tiles - tile0;
+    const uint32_t nvalid = left < (uint64_t)C::TPC ? (uint32_t)left : (uint32_t)C::TPC;
+    const uint32_t own = threadIdx.x / C::LPT;   // tile of the chunk this thread looks at first
+    const bool hi1 = a.mixed && own < nvalid && cur.is_hi(a, tile0 + own, own);
+    uint32_t chunk_bytes;
+    const uint64_t goff = (uint64_t)(C::G / 8) * ((uint64_t)a.lo * tile0 + hi_run);
 
-    float x[C::EPT];
-#pragma unroll
-    for (int o = 0; o < C::NOCT; ++o) {
-      float v[8];
-      load_oct<C>(stage, o, v);
-#pragma unroll
-      for (int k = 0; k < 8; ++k) x[8 * o + k] = v[k];
-    }
-
-    // Eq. 3: largest magnitude (first index), largest among the others
-    float a1 = fabsf(x[0]), a2 = 0.0f;
-    int d = 0;
-#pragma unroll
-    for (int k = 1; k < C::EPT; ++k) {
-      const float m = fabsf(x[k]);
-      const bool gt = m > a1;
-      a2 = gt ? a1 : fmaxf(a2, m);
-      d = gt ? k : d;
-      a1 = gt ? m : a1;
-    }
-    if constexpr (C::LPT == 2) {
-      const float o1 = __shfl_xor_sync(kFull, a1, 1), o2 = __shfl_xor_sync(kFull, a2, 1);
-      const int od = __shfl_xor_sync(kFull, d, 1);
-      const float l1 = half ? o1 : a1, l2 = half ? o2 : a2, u1 = half ? a1 : o1, u2 = half ? a2 : o2;
-      const int ld = half ? od : d, ud = half ? d : od;
-      const bool lw = l1 >= u1;   // the lower half holds the lower indices: it wins ties
-      a1 = lw ? l1 : u1;
-      a2 = lw ? fmaxf(l2, u1) : fmaxf(u2, l1);
-      d = lw ? ld : C::EPT + ud;
-    }
-    const float t1 = a2 + a.eps_ratio;
-    const float t2 = a.tau * t1;
-    const bool flag = a1 > t2;
-
-    // Eq. 4: pivot swap + Hadamard on flagged tiles
-    const unsigned fm = __ballot_sync(kFull, flag);
-    if (flag) {
-      if constexpr (C::LPT == 1) {
-        const float xd = load_elem<C>(stage, d), x0 = x[0];
-#pragma unroll
-        for (int k = 1; k < C::EPT; ++k) x[k] = (k == d) ? x0 : x[k];
-        x[0] = xd;
-        butterfly<C::EPT>(x);
+    if constexpr (C::LPT == 1) {
+      // ---- phase 1: thread r looks at tile r: outlier test (Eq. 3), then the CTA regroups its tiles
+      float a1, a2;
+      row_top2<C>(stage, (int)threadIdx.x, a1, a2);
+      const float t1 = a2 + a.eps_ratio;
+      const float t2 = a.tau * t1;
+      const bool flag1 = a1 > t2;
+      const Regroup rg = regroup((flag1 ? 2 : 0) | (hi1 ? 1 : 0), s_perm, s_cnt, [&](const Regroup &r) {
+        s_rowoff[threadIdx.x] = (uint16_t)((C::G / 8) * (a.lo * threadIdx.x + r.hi_before));
+        s_a1[threadIdx.x] = a1;
+        if ((threadIdx.x & 31) == 0) bitmap[tile0 / 32 + (threadIdx.x >> 5)] = r.hi_ballot;
+      });
+      chunk_bytes = (C::G / 8) * (a.lo * nvalid + rg.total_hi);
+      hi_run += rg.total_hi;
+      // ---- phase 2: this thread now owns tile `src` of the chunk
+      const int src = rg.src;
+      const bool flag = rg.cls & 2;
+      const uint32_t b = a.lo + (rg.cls & 1);
+      const uint64_t tile = tile0 + src;
+      const bool live = (uint32_t)src < nvalid;
+      uint32_t *dst = out + s_rowoff[src] / 4;
+      if (C::BF16 && !flag) {
+        const Quantiser q = encode_raw_bf16_row<C>(stage, src, b, dst, live);
+        if (live) { sz32[tile] = q.sz; pivot[tile] = 0; }
       } else {
+        float x[C::EPT];
+#pragma unroll
+        for (int o = 0; o < C::NOCT; ++o) {
+          float v[8];
+          load_oct<C>(stage, src, o, v);
+#pragma unroll
+          for (int k = 0; k < 8; ++k) x[8 * o + k] = v[k];
+        }
+        int d = 0;
+        if (flag) {   // Eq. 4: pivot swap + Hadamard
+          const float m = s_a1[src];
+#pragma unroll
+          for (int k = C::EPT - 1; k >= 0; --k) d = (fabsf(x[k]) == m) ? k : d;   // first index of the maximum
+          const float xd = load_elem<C>(stage, src, d), x0 = x[0];
+#pragma unroll
+          for (int k = 1; k < C::EPT; ++k) x[k] = (k == d) ? x0 : x[k];
+          x[0] = xd;
+          butterfly<C::EPT>(x);
+#pragma unroll
+          for (int k = 0; k < C::EPT; ++k) x[k] = x[k] * hadamard_scale<C>();
+        }
+        float mn = x[0], mx = x[0];
+#pragma unroll
+        for (int k = 1; k < C::EPT; ++k) { mn = fminf(mn, x[k]); mx = fmaxf(mx, x[k]); }
+        const Quantiser q = make_quantiser(mn, mx, b);
+        quantise_row<C::EPT>(x, mn, mx, q);
+        if (live) {
+          sz32[tile] = q.sz;
+          pivot[tile] = flag ? (uint8_t)(0x80 | d) : (uint8_t)0;
+          pack_row<C::EPT>([&](int k) { return x[k]; }, b, dst);
+        }
+      }
+    } else {
+      // ---- 128-wide tiles: two lanes per tile, no regrouping
+      const int half = threadIdx.x & 1;
+      const uint64_t tile = tile0 + own;
+      uint32_t hi_before, total_hi, tiles16;
+      pair_scan(hi1, reinterpret_cast<uint32_t *>(s_cnt), hi_before, total_hi, tiles16);
+      if ((threadIdx.x & 31) == 0)
+        reinterpret_cast<uint16_t *>(bitmap)[tile0 / 16 + (threadIdx.x >> 5)] = (uint16_t)tiles16;
+      chunk_bytes = (C::G / 8) * (a.lo * nvalid + total_hi);
+      hi_run += total_hi;
+      const uint32_t b = a.lo + (hi1 ? 1u : 0u);
+      const uint32_t row_off = (C::G / 8) * (a.lo * own + hi_before) + half * (C::EPT / 8) * b;
+      float x[C::EPT];
+#pragma unroll
+      for (int o = 0; o < C::NOCT; ++o) {
+        float v[8];
+        load_oct<C>(stage, (int)threadIdx.x, o, v);
+#pragma unroll
+        for (int k = 0; k < 8; ++k) x[8 * o + k] = v[k];
+      }
+      float a1 = fabsf(x[0]), a2 = 0.0f;
+      int d = 0;
+#pragma unroll
+      for (int k = 1; k < C::EPT; ++k) {
+        const float m = fabsf(x[k]);
+        const bool gt = m > a1;
+        a2 = gt ? a1 : fmaxf(a2, m);
+        d = gt ? k : d;
+        a1 = gt ? m : a1;
+      }
+      {
+        const float o1 = __shfl_xor_sync(kFull, a1, 1), o2 = __shfl_xor_sync(kFull, a2, 1);
+        const int od = __shfl_xor_sync(kFull, d, 1);
+        const float l1 = half ? o1 : a1, l2 = half ? o2 : a2, u1 = half ? a1 : o1, u2 = half ? a2 : o2;
+        const int ld = half ? od : d, ud = half ? d : od;
+        const bool lw = l1 >= u1;   // the lower half holds the lower indices: it wins ties
+        a1 = lw ? l1 : u1;
+        a2 = lw ? fmaxf(l2, u1) : fmaxf(u2, l1);
+        d = lw ? ld : C::EPT + ud;
+      }
+      const float t1 = a2 + a.eps_ratio;
+      const float t2 = a.tau * t1;
+      const bool flag = a1 > t2;
+      const unsigned fm = __ballot_sync(kFull, flag);
+      if (flag) {
         const int lane = threadIdx.x & 31, owner = d / C::EPT, dl = d % C::EPT;
         const float x0 = __shfl_sync(fm, x[0], lane & ~1);
-        const float xd = __shfl_sync(fm, load_elem<C>(stage, dl), (lane & ~1) + owner);
+        const float xd = __shfl_sync(fm, load_elem<C>(stage, (int)threadIdx.x, dl), (lane & ~1) + owner);
         if (half == owner) {
 #pragma unroll
           for (int k = 0; k < C::EPT; ++k) x[k] = (k == dl) ? x0 : x[k];
@@ -402,61 +725,35 @@ __global__ void __launch_bounds__(kThreads) quant_pack_kernel(const Args a) {
           const float p = __shfl_xor_sync(fm, x[k], 1);
           x[k] = half ? (p - x[k]) : (x[k] + p);
         }
+#pragma unroll
+        for (int k = 0; k < C::EPT; ++k) x[k] = x[k] * hadamard_scale<C>();
       }
-      constexpr float cG = (C::G == 32) ? 0.17677669529663687f : (C::G == 64) ? 0.125f : 0.08838834764831845f;
+      float mn = x[0], mx = x[0];
 #pragma unroll
-      for (int k = 0; k < C::EPT; ++k) x[k] = x[k] * cG;
-    }
-
-    // Sec. 3.3: min-max range -> binary16 zero-point and scale
-    float mn = x[0], mx = x[0];
-#pragma unroll
-    for (int k = 1; k < C::EPT; ++k) { mn = fminf(mn, x[k]); mx = fmaxf(mx, x[k]); }
-    if constexpr (C::LPT == 2) {
+      for (int k = 1; k < C::EPT; ++k) { mn = fminf(mn, x[k]); mx = fmaxf(mx, x[k]); }
       mn = fminf(mn, __shfl_xor_sync(kFull, mn, 1));
       mx = fmaxf(mx, __shfl_xor_sync(kFull, mx, 1));
-    }
-    const uint32_t b = a.lo + plan.is_hi;
-    const float qmax = (float)((1u << b) - 1u);
-    mn = mn + 0.0f;
-    mn = fminf(fmaxf(mn, -65504.0f), 65504.0f);
-    const __half zh = __float2half_rn(mn);
-    const float z = __half2float(zh);
-    float s = __fdiv_rn(mx - z, qmax);
-    s = (s > 0.0f) ? s : 0.0f;
-    s = fminf(s, 65504.0f);
-    const __half sh = __float2half_rn(s);
-    const float sf = __half2float(sh);
-    const float inv_s = sf > 0.0f ? __fdiv_rn(1.0f, sf) : 0.0f;
-
-    // q = rint(clamp((v - z) * inv_s, 0, qmax)); adding 1.5*2^23 rounds to nearest-even
-    uint32_t code[C::EPT];
-#pragma unroll
-    for (int k = 0; k < C::EPT; ++k) {
-      float y = (x[k] - z) * inv_s;
-      y = fminf(fmaxf(y, 0.0f), qmax);
-      code[k] = __float_as_uint(y + 12582912.0f) & 0x1ffu;
-    }
-
-    if (valid) {
-      if (half == 0) {
-        sz32[tile] = (uint32_t)__half_as_ushort(sh) | ((uint32_t)__half_as_ushort(zh) << 16);
-        pivot[tile] = flag ? (uint8_t)(0x80 | d) : (uint8_t)0;
-      }
-      uint32_t *dst = out + plan.row_off / 4;
-      switch (b) {
-        case 2: pack_store<C, 2>(code, dst); break;
-        case 3: pack_store<C, 3>(code, dst); break;
-        case 4: pack_store<C, 4>(code, dst); break;
-        case 5: pack_store<C, 5>(code, dst); break;
-        case 6: pack_store<C, 6>(code, dst); break;
-        case 7: pack_store<C, 7>(code, dst); break;
-        default: pack_store<C, 8>(code, dst); break;
+      const Quantiser q = make_quantiser(mn, mx, b);
+      quantise_row<C::EPT>(x, mn, mx, q);
+      if (own < nvalid) {
+        if (half == 0) {
+          sz32[tile] = q.sz;
+          pivot[tile] = flag ? (uint8_t)(0x80 | d) : (uint8_t)0;
+        }
+        pack_row<C::EPT>([&](int k) { return x[k]; }, b, out + row_off / 4);
       }
     }
+    cur.advance(a, C::TPC);
     __syncthreads();
-    uint32_t *gdst = reinterpret_cast<uint32_t *>(a.packed + a.off_payload + plan.goff);
-    for (uint32_t i = threadIdx.x; i < plan.bytes / 4; i += kThreads) gdst[i] = out[i];
+    // the chunk's codes leave with coalesced stores (payload offsets are multiples of G/8 bytes)
+    if constexpr (C::G >= 64) {
+      uint2 *gdst = reinterpret_cast<uint2 *>(a.packed + a.off_payload + goff);
+      const uint2 *s2 = reinterpret_cast<const uint2 *>(out);
+      for (uint32_t i = threadIdx.x; i < chunk_bytes / 8; i += kThreads) gdst[i] = s2[i];
+    } else {
+      uint32_t *gdst = reinterpret_cast<uint32_t *>(a.packed + a.off_payload + goff);
+      for (uint32_t i = threadIdx.x; i < chunk_bytes / 4; i += kThreads) gdst[i] = out[i];
+    }
   });
 }
 
@@ -464,104 +761,182 @@ __global__ void __launch_bounds__(kThreads) quant_pack_kernel(const Args a) {
 // Decode
 // ------------------------------------------------------------------------------------------
 
-// hi tiles per 128 tiles, straight from the received bit map; CTA 0 also checks the header.
-__global__ void __launch_bounds__(kThreads) count_kernel(const Args a) {
-  const uint64_t n128 = (a.n_tiles + 127) / 128;
-  const uint64_t i = (uint64_t)blockIdx.x * kThreads + threadIdx.x;
-  if (blockIdx.x == 0 && threadIdx.x < 32) {
-    const uint32_t got = reinterpret_cast<const uint32_t *>(a.packed)[threadIdx.x];
-    // seed / rounding / constants are part of the header, so a buffer from another configuration is refused
-    if (got != a.header[threadIdx.x]) atomicOr(a.status, 1u /* TAHQ_DEV_BAD_HEADER */);
-  }
-  if (i >= n128) return;
-  uint32_t n = 0;
-  if (a.mixed) {
-    const uint32_t *bm = reinterpret_cast<const uint32_t *>(a.packed + a.off_bitmap) + i * 4;
+template <int N>
+__device__ __forceinline__ void load_dequant(const uint32_t *src, uint32_t bits, float s, float z, float (&x)[N]) {
+  uint32_t w[N / 4];
+  if constexpr (N == 64) {   // 64-wide rows start on 8-byte boundaries
 #pragma unroll
-    for (int w = 0; w < 4; ++w) {
-      const uint64_t first = i * 128 + 32ull * w;
-      if (first < a.n_tiles) {
-        const uint64_t left = a.n_tiles - first;
-        n += __popc(bm[w] & (left >= 32 ? 0xffffffffu : ((1u << (uint32_t)left) - 1u)));
-      }
+    for (int j = 0; j < N / 8; ++j) {
+      uint2 v = make_uint2(0u, 0u);
+      if (j < (int)(N * bits / 64)) v = __ldg(reinterpret_cast<const uint2 *>(src) + j);
+      w[2 * j] = v.x; w[2 * j + 1] = v.y;
     }
+  } else {
+#pragma unroll
+    for (int j = 0; j < N / 4; ++j) w[j] = (j < (int)(N * bits / 32)) ? __ldg(src + j) : 0u;
   }
-  a.cnt128[i] = n;
+  switch (bits) {
+    case 2: unpack_dequant<2, N>(w, s, z, x); break;
+    case 3: unpack_dequant<3, N>(w, s, z, x); break;
+    case 4: unpack_dequant<4, N>(w, s, z, x); break;
+    case 5: unpack_dequant<5, N>(w, s, z, x); break;
+    case 6: unpack_dequant<6, N>(w, s, z, x); break;
+    case 7: unpack_dequant<7, N>(w, s, z, x); break;
+    default: unpack_dequant<8, N>(w, s, z, x); break;
+  }
 }
 
-template <class C, int W>
-__device__ __forceinline__ void load_unpack(const uint32_t *src, uint32_t (&code)[C::EPT]) {
-  uint32_t w[C::EPT * W / 32];
+// Store a register row into the swizzled output stage (narrowing to bf16 with round-to-nearest-even).
+template <class C>
+__device__ __forceinline__ void stage_row(uint8_t *stage, int row, const float (&x)[C::EPT]) {
+  if constexpr (C::BF16) {
 #pragma unroll
-  for (int j = 0; j < C::EPT * W / 32; ++j) w[j] = __ldg(src + j);
-  unpack_words<W, C::EPT>(w, code);
+    for (int q = 0; q < C::CPR; ++q) {
+      uint32_t u[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const __nv_bfloat162 h2 = __floats2bfloat162_rn(x[8 * q + 2 * j], x[8 * q + 2 * j + 1]);
+        u[j] = *reinterpret_cast<const uint32_t *>(&h2);
+      }
+      *reinterpret_cast<uint4 *>(stage + (size_t)phys_chunk<C>(row, q) * 16) = make_uint4(u[0], u[1], u[2], u[3]);
+    }
+  } else {
+#pragma unroll
+    for (int q = 0; q < C::CPR; ++q)
+      *reinterpret_cast<float4 *>(stage + (size_t)phys_chunk<C>(row, q) * 16) =
+          make_float4(x[4 * q], x[4 * q + 1], x[4 * q + 2], x[4 * q + 3]);
+  }
 }
 
 template <class C>
-__global__ void __launch_bounds__(kThreads) decode_kernel(const Args a) {
+__global__ void __launch_bounds__(kThreads, 2) decode_kernel(const Args a) {
   extern __shared__ __align__(128) uint8_t smem[];   // one swizzled output stage
-  if (*reinterpret_cast<volatile uint32_t *>(a.status) != 0) return;   // refused buffer: leave the output alone
+  __shared__ uint8_t s_perm[kThreads];
+  __shared__ uint2 s_cnt[kThreads / 32];
+  __shared__ uint16_t s_rowoff[kThreads];
+  __shared__ uint8_t s_pv[kThreads];
+  __shared__ uint32_t s_bad;
   const uint32_t *sz32 = reinterpret_cast<const uint32_t *>(a.packed + a.off_sz);
   const uint8_t *pivot = a.packed + a.off_pivot;
+  const uint32_t *bitmap = reinterpret_cast<const uint32_t *>(a.packed + a.off_bitmap);
   const uint64_t n_chunks = (a.n_tiles + C::TPC - 1) / C::TPC;
-  for (uint64_t c = blockIdx.x; c < n_chunks; c += gridDim.x) {
-    const uint64_t tile0 = c * C::TPC;
-    const int half = threadIdx.x % C::LPT;
-    const uint64_t tile = tile0 + threadIdx.x / C::LPT;
-    const bool valid = tile < a.n_tiles;
-    const ChunkPlan<C> plan = plan_chunk<C>(a, c);
-    const uint32_t b = a.lo + plan.is_hi;
+  uint64_t c0, c1;
+  cta_chunk_range(n_chunks, c0, c1);
 
-    float x[C::EPT];
-    uint32_t pv = 0;
-    if (valid) {
-      const uint32_t szw = __ldg(sz32 + tile);
-      const float s = __half2float(__ushort_as_half((unsigned short)(szw & 0xffffu)));
-      const float z = __half2float(__ushort_as_half((unsigned short)(szw >> 16)));
-      pv = __ldg(pivot + tile);
-      const uint32_t *src = reinterpret_cast<const uint32_t *>(a.packed + a.off_payload + plan.goff + plan.row_off);
-      uint32_t code[C::EPT];
-      switch (b) {
-        case 2: load_unpack<C, 2>(src, code); break;
-        case 3: load_unpack<C, 3>(src, code); break;
-        case 4: load_unpack<C, 4>(src, code); break;
-        case 5: load_unpack<C, 5>(src, code); break;
-        case 6: load_unpack<C, 6>(src, code); break;
-        case 7: load_unpack<C, 7>(src, code); break;
-        default: load_unpack<C, 8>(src, code); break;
+  // CTA 0 compares the received header with the one these parameters produce; its verdict travels
+  // with the offset prefix, so a refused buffer leaves the output untouched.
+  bool refuse = false;
+  if (blockIdx.x == 0) {
+    if (threadIdx.x == 0) s_bad = 0;
+    __syncthreads();
+    if (threadIdx.x < 32 && reinterpret_cast<const uint32_t *>(a.packed)[threadIdx.x] != a.header[threadIdx.x]) s_bad = 1;
+    __syncthreads();
+    refuse = s_bad != 0;
+    if (refuse && threadIdx.x == 0) atomicOr(a.status, 1u /* TAHQ_DEV_BAD_HEADER */);
+  }
+  // higher-width tiles before this CTA's range (Sec. 3.4 offsets), counted from the received bit map
+  uint64_t hi_run = 0;
+  {
+    uint32_t n = 0;
+    if (a.mixed && !refuse) {
+      const uint64_t t0 = c0 * C::TPC, t1 = c1 * C::TPC < a.n_tiles ? c1 * C::TPC : a.n_tiles;
+      for (uint64_t wi = t0 / 32 + threadIdx.x; wi * 32 < t1; wi += kThreads) {
+        const uint64_t leftw = t1 - wi * 32;
+        n += __popc(__ldg(bitmap + wi) & (leftw >= 32 ? 0xffffffffu : ((1u << (uint32_t)leftw) - 1u)));
       }
-#pragma unroll
-      for (int k = 0; k < C::EPT; ++k) x[k] = __fmaf_rn((float)code[k], s, z);
-    } else {
-#pragma unroll
-      for (int k = 0; k < C::EPT; ++k) x[k] = 0.0f;
     }
+    const uint32_t mine = block_sum(n);
+    bool stop;
+    hi_run = cta_exclusive_prefix(a, mine, refuse, stop);
+    if (blockIdx.x == gridDim.x - 1 && threadIdx.x == 0 && a.mixed && !stop &&
+        hi_run + mine != a.n_groups * a.k_hi)
+      atomicOr(a.status, 2u /* TAHQ_DEV_BAD_BITMAP */);
+    if (stop) return;
+  }
 
-    const bool flag = (pv & 0x80u) != 0;
-    const unsigned fm = __ballot_sync(kFull, flag);
-    if (flag) {
-      const int d = pv & 0x7f;
-      butterfly<C::EPT>(x);
-      if constexpr (C::LPT == 2) {
+  for (uint64_t c = c0; c < c1; ++c) {
+    const uint64_t tile0 = c * C::TPC;
+    const uint64_t left = a.n_tiles - tile0;
+    const uint32_t nvalid = left < (uint64_t)C::TPC ? (uint32_t)left : (uint32_t)C::TPC;
+    const uint32_t own = threadIdx.x / C::LPT;
+    const uint64_t goff = (uint64_t)(C::G / 8) * ((uint64_t)a.lo * tile0 + hi_run);
+    const uint8_t *pay = a.packed + a.off_payload + goff;
+    float x[C::EPT];
+    bool hi1 = false;
+    if (a.mixed && own < nvalid) hi1 = (__ldg(bitmap + (tile0 + own) / 32) >> ((tile0 + own) & 31)) & 1u;
+    uint32_t chunk_bytes;
+
+    if constexpr (C::LPT == 1) {
+      // phase 1: thread r reads tile r's pivot byte; the CTA regroups tiles by (transformed?, width)
+      const uint32_t pv1 = own < nvalid ? __ldg(pivot + tile0 + own) : 0u;
+      const Regroup rg = regroup(((pv1 & 0x80u) ? 2 : 0) | (hi1 ? 1 : 0), s_perm, s_cnt, [&](const Regroup &r) {
+        s_rowoff[threadIdx.x] = (uint16_t)((C::G / 8) * (a.lo * threadIdx.x + r.hi_before));
+        s_pv[threadIdx.x] = (uint8_t)pv1;
+      });
+      chunk_bytes = (C::G / 8) * (a.lo * nvalid + rg.total_hi);
+      hi_run += rg.total_hi;
+      const bool fits = goff + chunk_bytes <= a.payload_bytes;   // false only for a corrupt bit map
+      // phase 2
+      const int src = rg.src;
+      const bool flag = rg.cls & 2;
+      const uint32_t b = a.lo + (rg.cls & 1);
+      const uint64_t tile = tile0 + src;
+      if ((uint32_t)src < nvalid && fits) {
+        const uint32_t szw = __ldg(sz32 + tile);
+        const float s = __half2float(__ushort_as_half((unsigned short)(szw & 0xffffu)));
+        const float z = __half2float(__ushort_as_half((unsigned short)(szw >> 16)));
+        load_dequant<C::EPT>(reinterpret_cast<const uint32_t *>(pay + s_rowoff[src]), b, s, z, x);
+      } else {
 #pragma unroll
-        for (int k = 0; k < C::EPT; ++k) {
-          const float p = __shfl_xor_sync(fm, x[k], 1);
-          x[k] = half ? (p - x[k]) : (x[k] + p);
-        }
+        for (int k = 0; k < C::EPT; ++k) x[k] = 0.0f;
       }
-      constexpr float cG = (C::G == 32) ? 0.17677669529663687f : (C::G == 64) ? 0.125f : 0.08838834764831845f;
+      if (flag) {
+        const int d = s_pv[src] & 0x7f;
+        butterfly<C::EPT>(x);
 #pragma unroll
-      for (int k = 0; k < C::EPT; ++k) x[k] = x[k] * cG;
-      // un-swap coordinates 0 and d
-      if constexpr (C::LPT == 1) {
-        float xd = x[0];
+        for (int k = 0; k < C::EPT; ++k) x[k] = x[k] * hadamard_scale<C>();
+        float xd = x[0];   // un-swap coordinates 0 and d
 #pragma unroll
         for (int k = 1; k < C::EPT; ++k) xd = (k == d) ? x[k] : xd;
         const float x0 = x[0];
 #pragma unroll
         for (int k = 1; k < C::EPT; ++k) x[k] = (k == d) ? x0 : x[k];
         x[0] = xd;
+      }
+      stage_row<C>(smem, src, x);
+    } else {
+      const int half = threadIdx.x & 1;
+      const uint64_t tile = tile0 + own;
+      uint32_t hi_before, total_hi, tiles16;
+      pair_scan(hi1, reinterpret_cast<uint32_t *>(s_cnt), hi_before, total_hi, tiles16);
+      chunk_bytes = (C::G / 8) * (a.lo * nvalid + total_hi);
+      hi_run += total_hi;
+      const bool fits = goff + chunk_bytes <= a.payload_bytes;
+      const uint32_t b = a.lo + (hi1 ? 1u : 0u);
+      const uint32_t row_off = (C::G / 8) * (a.lo * own + hi_before) + half * (C::EPT / 8) * b;
+      uint32_t pv = 0;
+      if (own < nvalid && fits) {
+        const uint32_t szw = __ldg(sz32 + tile);
+        const float s = __half2float(__ushort_as_half((unsigned short)(szw & 0xffffu)));
+        const float z = __half2float(__ushort_as_half((unsigned short)(szw >> 16)));
+        pv = __ldg(pivot + tile);
+        load_dequant<C::EPT>(reinterpret_cast<const uint32_t *>(pay + row_off), b, s, z, x);
       } else {
+#pragma unroll
+        for (int k = 0; k < C::EPT; ++k) x[k] = 0.0f;
+      }
+      const bool flag = (pv & 0x80u) != 0;
+      const unsigned fm = __ballot_sync(kFull, flag);
+      if (flag) {
+        const int d = pv & 0x7f;
+        butterfly<C::EPT>(x);
+#pragma unroll
+        for (int k = 0; k < C::EPT; ++k) {
+          const float p = __shfl_xor_sync(fm, x[k], 1);
+          x[k] = half ? (p - x[k]) : (x[k] + p);
+        }
+#pragma unroll
+        for (int k = 0; k < C::EPT; ++k) x[k] = x[k] * hadamard_scale<C>();
         const int lane = threadIdx.x & 31, owner = d / C::EPT, dl = d % C::EPT;
         float mine = x[0];
 #pragma unroll
@@ -574,32 +949,12 @@ __global__ void __launch_bounds__(kThreads) decode_kernel(const Args a) {
         }
         if (half == 0) x[0] = xd;
       }
+      stage_row<C>(smem, (int)threadIdx.x, x);
     }
 
-    // stage the row (swizzled), then write the chunk out with coalesced 16-byte stores
-    const int row = threadIdx.x;
-    if constexpr (C::BF16) {
-#pragma unroll
-      for (int q = 0; q < C::CPR; ++q) {
-        uint4 w;
-        uint32_t u[4];
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          const __nv_bfloat162 h2 = __floats2bfloat162_rn(x[8 * q + 2 * j], x[8 * q + 2 * j + 1]);
-          u[j] = *reinterpret_cast<const uint32_t *>(&h2);
-        }
-        w.x = u[0]; w.y = u[1]; w.z = u[2]; w.w = u[3];
-        *reinterpret_cast<uint4 *>(smem + (size_t)phys_chunk<C>(row, q) * 16) = w;
-      }
-    } else {
-#pragma unroll
-      for (int q = 0; q < C::CPR; ++q)
-        *reinterpret_cast<float4 *>(smem + (size_t)phys_chunk<C>(row, q) * 16) =
-            make_float4(x[4 * q], x[4 * q + 1], x[4 * q + 2], x[4 * q + 3]);
-    }
+    // the chunk leaves with coalesced 16-byte stores
     __syncthreads();
-    const uint64_t left = a.n_tiles - tile0;
-    const uint32_t valid_bytes = (uint32_t)(left < (uint64_t)C::TPC ? left : (uint64_t)C::TPC) * C::G * C::ESZ;
+    const uint32_t valid_bytes = nvalid * C::G * C::ESZ;
     uint8_t *gout = a.out + tile0 * (uint64_t)(C::G * C::ESZ);
 #pragma unroll
     for (int i = 0; i < C::CPR; ++i) {
