@@ -304,22 +304,30 @@ void tahqo_philox4x32_10(const uint32_t key[2], const uint32_t ctr[4], uint32_t 
 }
 
 /* q_k = clamp(round((v_k - z) / s), 0, 2^b - 1), the division done as a
- * multiplication by the binary32 reciprocal of the stored scale.
- * rounding 0: round-half-even.  rounding 1: floor(y + u), u uniform in [0,1)
- * with 24 bits, taken from word (i mod 4) of Philox(key = seed, counter = i/4)
- * where i = first_elem + k is the element's index in the whole tensor. */
+ * multiplication by the binary32 reciprocal of the stored scale.  The
+ * difference d = v_k - z is a binary32 subtraction; the product d * inv_s is
+ * taken EXACTLY (two binary32 factors multiply exactly in binary64) and rounded
+ * once, to the nearest integer, ties to even.
+ * rounding 0: as above.  rounding 1: floor(y + u) on the binary32 product y,
+ * u uniform in [0,1) with 24 bits, taken from word (i mod 4) of
+ * Philox(key = seed, counter = i/4) where i = first_elem + k is the element's
+ * index in the whole tensor. */
 void tahqo_quantise(const float *v, uint32_t G, uint32_t bits, uint16_t s_h, uint16_t z_h,
                     uint32_t rounding, uint64_t seed, uint64_t first_elem, uint32_t *q) {
   float s = tahqo_f16_to_f32(s_h), z = tahqo_f16_to_f32(z_h);
   float inv_s = s > 0.0f ? 1.0f / s : 0.0f;
   float qmax = (float)((1u << bits) - 1u);
   for (uint32_t k = 0; k < G; k++) {
-    float y = (v[k] - z) * inv_s;
-    if (!(y > 0.0f)) y = 0.0f;
-    if (y > qmax) y = qmax;
+    float d = v[k] - z;
     if (rounding == 0) {
-      q[k] = (uint32_t)rintf(y);                 /* default rounding mode: nearest, ties to even */
+      double y = (double)d * (double)inv_s;       /* exact */
+      if (!(y > 0.0)) y = 0.0;
+      if (y > (double)qmax) y = (double)qmax;
+      q[k] = (uint32_t)rint(y);                    /* default rounding mode: nearest, ties to even */
     } else {
+      float y = d * inv_s;
+      if (!(y > 0.0f)) y = 0.0f;
+      if (y > qmax) y = qmax;
       uint64_t i = first_elem + k, c = i / 4;
       uint32_t key[2] = { (uint32_t)seed, (uint32_t)(seed >> 32) };
       uint32_t ctr[4] = { (uint32_t)c, (uint32_t)(c >> 32), 0u, 0u };

@@ -155,7 +155,7 @@ def test_tau_inf_integer_budget_is_plain_group_quantisation():
         qmax = np.float32(2 ** bits - 1)
         z = t.min(axis=1, keepdims=True).astype(np.float16).astype(np.float32)
         s = ((t.max(axis=1, keepdims=True) - z) / qmax).astype(np.float16).astype(np.float32)
-        q = np.clip(np.rint((t - z) * (np.float32(1) / s)), 0, qmax)
+        q = np.clip(np.rint((t - z).astype(np.float64) * (np.float32(1) / s).astype(np.float64)), 0, qmax)
         want = (q.astype(np.float64) * s.astype(np.float64) + z.astype(np.float64)).astype(np.float32)  # one rounding
         assert np.array_equal(y.reshape(-1, 64), want)
 

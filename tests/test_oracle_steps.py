@@ -250,7 +250,8 @@ def test_quantiser_is_textbook_minmax(bits):
         assert zh == int(np.float16(v.min()).view(np.uint16))
         assert sh == int(np.float16(s).view(np.uint16))
         q = O.quantise(v, bits, sh, zh)
-        want = np.clip(np.rint((v - z) * (np.float32(1) / s)), 0, qmax).astype(np.uint32)
+        # difference in binary32, product with the binary32 reciprocal taken exactly, one rounding
+        want = np.clip(np.rint((v - z).astype(np.float64) * np.float64(np.float32(1) / s)), 0, qmax).astype(np.uint32)
         assert np.array_equal(q, want)
         # error bound: half a step plus the binary16 rounding of z and s
         xhat = z + q.astype(np.float32) * s
