@@ -85,8 +85,7 @@ static tahq_status make_plan(const tahq_params *p, Plan *pl) {
   pl->cpg = 1;
   pl->cand_cap = 0;
   if (pl->mixed && !pl->direct) {
-    uint64_t cpg = (L.tiles_per_group + 16383) / 16384;
-    pl->cpg = (uint32_t)(cpg > 64 ? 64 : cpg);
+    pl->cpg = (uint32_t)((L.tiles_per_group + kSelSlice - 1) / kSelSlice);
     pl->cand_cap = (uint32_t)(L.tiles_per_group < 32768 ? L.tiles_per_group : 32768);
   }
   const bool hist = pl->mixed && !pl->direct;
@@ -180,7 +179,7 @@ static int prepare(K kernel, int smem, const DevInfo &d, std::atomic<int> *cache
 }
 
 template <class C> struct Stages {
-  static constexpr int STATS = (C::ROWB == 256) ? 2 : (C::ROWB == 128 ? 3 : 4);
+  static constexpr int STATS = (C::ROWB == 64) ? 3 : 2;
   static constexpr int QUANT = (C::ROWB == 256) ? 2 : (C::ROWB == 128 ? 2 : 3);
 };
 
@@ -212,7 +211,7 @@ static tahq_status encode_t(const Plan &pl, const Args &a, cudaStream_t st) {
     TAHQ_LAUNCH("select", st, select_kernel<<<(unsigned)(a.n_groups * a.cpg), kSelThreads, sel_smem, st>>>(a));
   }
   constexpr int NQ = Stages<C>::QUANT;
-  const int smem = NQ * C::STAGE_BYTES + C::MAX_PAY;
+  const int smem = NQ * C::STAGE_BYTES;
   const int occ = prepare(quant_pack_kernel<C, NQ>, smem, d, occ_quant);
   if (!occ) return TAHQ_ERR_CUDA;
   TAHQ_LAUNCH("quant_pack", st,

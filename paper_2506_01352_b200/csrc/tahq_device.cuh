@@ -67,15 +67,19 @@ __device__ __forceinline__ void cp_async_wait() {
 template <class C>
 __device__ __forceinline__ void issue_chunk(const uint8_t *in, uint64_t n_tiles, uint64_t c, uint8_t *stage) {
   const uint64_t tile0 = c * C::TPC;
-  const uint64_t rem = n_tiles - tile0;
-  const uint32_t valid_bytes = (uint32_t)(rem < (uint64_t)C::TPC ? rem : (uint64_t)C::TPC) * C::G * C::ESZ;
-  const uint8_t *src = in + tile0 * (uint64_t)(C::G * C::ESZ);
+  const uint8_t *src = in + tile0 * (uint64_t)(C::G * C::ESZ) + (size_t)threadIdx.x * 16;
+  // chunk index ci = i*kThreads + tid lies in row ci / CPR, whose swizzle depends on tid only
+  uint8_t *dst = stage + (size_t)((int)threadIdx.x ^ swz<C>((int)threadIdx.x / C::CPR)) * 16;
+  if (tile0 + C::TPC <= n_tiles) {
 #pragma unroll
-  for (int i = 0; i < C::CPR; ++i) {
-    const int ci = i * kThreads + (int)threadIdx.x;
-    const int row = ci / C::CPR;
-    const bool ok = (uint32_t)ci * 16u < valid_bytes;
-    cp_async16(stage + (size_t)(ci ^ swz<C>(row)) * 16, ok ? src + (size_t)ci * 16 : src, ok ? 16 : 0);
+    for (int i = 0; i < C::CPR; ++i) cp_async16(dst + (size_t)i * kThreads * 16, src + (size_t)i * kThreads * 16, 16);
+  } else {
+    const uint32_t valid_bytes = (uint32_t)(n_tiles - tile0) * C::G * C::ESZ;
+#pragma unroll
+    for (int i = 0; i < C::CPR; ++i) {
+      const bool ok = (uint32_t)(i * kThreads + (int)threadIdx.x) * 16u < valid_bytes;
+      cp_async16(dst + (size_t)i * kThreads * 16, ok ? src + (size_t)i * kThreads * 16 : in, ok ? 16 : 0);
+    }
   }
 }
 
@@ -108,6 +112,38 @@ __device__ __forceinline__ float load_elem(const uint8_t *stage, int row, int k)
 }
 
 // ------------------------------------------------------------------------------------------
+// bf16 pairs handled in their packed form (sm_100a: packed bf16 min/max run on the ALU pipe, one
+// instruction per two elements; a bf16 operand can feed an fp32 add on the FMA pipe directly)
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t bf2_max_abs(uint32_t a, uint32_t b) {   // magnitudes; sign bits are garbage
+  uint32_t d;
+  asm("max.xorsign.abs.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+  return d;
+}
+__device__ __forceinline__ uint32_t bf2_min_abs(uint32_t a, uint32_t b) {
+  uint32_t d;
+  asm("min.xorsign.abs.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+  return d;
+}
+__device__ __forceinline__ uint32_t bf2_max(uint32_t a, uint32_t b) {
+  uint32_t d;
+  asm("max.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+  return d;
+}
+__device__ __forceinline__ uint32_t bf2_min(uint32_t a, uint32_t b) {
+  uint32_t d;
+  asm("min.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+  return d;
+}
+// (lo + c, hi + c) in binary32 for the two bf16 halves of w: the widening is exact, so this equals
+// widening first and adding afterwards; with c = -0.0f it is the widening itself.
+__device__ __forceinline__ void bf2_add_f32(uint32_t w, float c, float &lo, float &hi) {
+  asm("{\n\t.reg .b16 l, h;\n\tmov.b32 {l, h}, %2;\n\tadd.rn.f32.bf16 %0, l, %3;\n\tadd.rn.f32.bf16 %1, h, %3;\n\t}"
+      : "=f"(lo), "=f"(hi)
+      : "r"(w), "f"(c));
+}
+
+// ------------------------------------------------------------------------------------------
 // Arithmetic of Eq. 1-2 (binary32, fixed order; the library is compiled with -fmad=false so that
 // only the fused multiply-adds written here are fused)
 // ------------------------------------------------------------------------------------------
@@ -126,45 +162,114 @@ __device__ __forceinline__ float tree(float (&t)[N]) {
   return t[0];
 }
 
-// log2 of a positive normal number: exponent + u*Q(u), u = mantissa - 1, Q of degree 5.
-__device__ __forceinline__ float lg2_poly(float x) {
-  const uint32_t xi = __float_as_uint(x);
-  const float e = (float)((int)(xi >> 23) - 127);
-  const float u = __uint_as_float((xi & 0x007fffffu) | 0x3f800000u) - 1.0f;
-  float q = -0x1.a762d6p-6f;
-  q = __fmaf_rn(q, u, 0x1.f2e252p-4f);
-  q = __fmaf_rn(q, u, -0x1.1c9334p-2f);
-  q = __fmaf_rn(q, u, 0x1.d487c6p-2f);
-  q = __fmaf_rn(q, u, -0x1.6fb0bcp-1f);
-  q = __fmaf_rn(q, u, 0x1.714aa0p+0f);
-  return __fmaf_rn(u, q, e);
+// Pairs of binary32 values processed by one instruction (sm_100a add/mul/fma .f32x2: IEEE
+// round-to-nearest per lane, so results equal the scalar operations bit for bit).  The assembler
+// contracts a packed multiply that feeds a packed add into one packed fma even with explicit .rn
+// and --fmad=false, which changes the rounding; so no result of mul2 may be an operand of add2
+// (or the addend of fma2): such products are formed with scalar multiplies instead.
+__device__ __forceinline__ float2 f2(float a, float b) { return make_float2(a, b); }
+__device__ __forceinline__ float2 f2(float a) { return make_float2(a, a); }
+__device__ __forceinline__ float2 add2(float2 a, float2 b) {
+  float2 d;
+  asm("add.rn.f32x2 %0, %1, %2;"
+      : "=l"(reinterpret_cast<unsigned long long &>(d))
+      : "l"(reinterpret_cast<const unsigned long long &>(a)), "l"(reinterpret_cast<const unsigned long long &>(b)));
+  return d;
+}
+__device__ __forceinline__ float2 mul2(float2 a, float2 b) {
+  float2 d;
+  asm("mul.rn.f32x2 %0, %1, %2;"
+      : "=l"(reinterpret_cast<unsigned long long &>(d))
+      : "l"(reinterpret_cast<const unsigned long long &>(a)), "l"(reinterpret_cast<const unsigned long long &>(b)));
+  return d;
+}
+__device__ __forceinline__ float2 fma2(float2 a, float2 b, float2 c) {
+  float2 d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;"
+      : "=l"(reinterpret_cast<unsigned long long &>(d))
+      : "l"(reinterpret_cast<const unsigned long long &>(a)), "l"(reinterpret_cast<const unsigned long long &>(b)),
+        "l"(reinterpret_cast<const unsigned long long &>(c)));
+  return d;
+}
+
+// log2 of positive normal numbers: exponent + u*Q(u), u = mantissa - 1, Q of degree 5.
+__device__ __forceinline__ float2 lg2_poly2(float2 x) {
+  const uint32_t x0 = __float_as_uint(x.x), x1 = __float_as_uint(x.y);
+  const float2 e = add2(f2((float)(int)(x0 >> 23), (float)(int)(x1 >> 23)), f2(-127.0f));
+  const float2 m = f2(__uint_as_float((x0 & 0x007fffffu) | 0x3f800000u), __uint_as_float((x1 & 0x007fffffu) | 0x3f800000u));
+  const float2 u = add2(m, f2(-1.0f));
+  float2 q = f2(-0x1.a762d6p-6f);
+  q = fma2(q, u, f2(0x1.f2e252p-4f));
+  q = fma2(q, u, f2(-0x1.1c9334p-2f));
+  q = fma2(q, u, f2(0x1.d487c6p-2f));
+  q = fma2(q, u, f2(-0x1.6fb0bcp-1f));
+  q = fma2(q, u, f2(0x1.714aa0p+0f));
+  return fma2(u, q, e);
+}
+
+// neighbours-first pairwise tree over 8 pairs (each lane of the pair is its own sum)
+__device__ __forceinline__ float2 tree8x2(const float2 (&v)[8]) {
+  const float2 a = add2(v[0], v[1]), b = add2(v[2], v[3]);
+  const float2 c = add2(v[4], v[5]), d = add2(v[6], v[7]);
+  return add2(add2(a, b), add2(c, d));
+}
+
+// Magnitudes of octs 2p and 2p+1 of a row, element k of both octs in one pair.
+template <class C>
+__device__ __forceinline__ void load_abs_oct_pair(const uint8_t *stage, int row, int p, float2 (&a)[8]) {
+  if constexpr (C::BF16) {
+    const uint4 w0 = *reinterpret_cast<const uint4 *>(stage + (size_t)phys_chunk<C>(row, 2 * p) * 16);
+    const uint4 w1 = *reinterpret_cast<const uint4 *>(stage + (size_t)phys_chunk<C>(row, 2 * p + 1) * 16);
+    const uint32_t u0[4] = {w0.x, w0.y, w0.z, w0.w}, u1[4] = {w1.x, w1.y, w1.z, w1.w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      float l0, h0, l1, h1;   // clearing the sign bits of the packed word, then widening on the FMA pipe
+      bf2_add_f32(u0[j] & 0x7fff7fffu, -0.0f, l0, h0);
+      bf2_add_f32(u1[j] & 0x7fff7fffu, -0.0f, l1, h1);
+      a[2 * j] = f2(l0, l1);
+      a[2 * j + 1] = f2(h0, h1);
+    }
+  } else {
+    float v0[8], v1[8];
+    load_oct<C>(stage, row, 2 * p, v0);
+    load_oct<C>(stage, row, 2 * p + 1, v1);
+#pragma unroll
+    for (int k = 0; k < 8; ++k) a[k] = f2(fabsf(v0[k]), fabsf(v1[k]));
+  }
 }
 
 // Entropy score of the tile this thread (pair) owns: -sum p log2(p + varsigma), p = |a| / (L1 + eps).
 template <class C>
 __device__ __forceinline__ float tile_score(const uint8_t *stage, float eps_l1, float eps_log) {
+  constexpr int NP = C::NOCT / 2;
+  const int row = (int)threadIdx.x;
+  float2 a[NP][8];
   float part[C::NOCT];
 #pragma unroll
-  for (int o = 0; o < C::NOCT; ++o) {
-    float v[8];
-    load_oct<C>(stage, (int)threadIdx.x, o, v);
-#pragma unroll
-    for (int k = 0; k < 8; ++k) v[k] = fabsf(v[k]);
-    part[o] = tree8(v);
+  for (int p = 0; p < NP; ++p) {
+    load_abs_oct_pair<C>(stage, row, p, a[p]);
+    const float2 s = tree8x2(a[p]);
+    part[2 * p] = s.x;
+    part[2 * p + 1] = s.y;
   }
   float L1 = tree<C::NOCT>(part);
   if constexpr (C::LPT == 2) L1 = L1 + __shfl_xor_sync(kFull, L1, 1);
   const float inv = __fdiv_rn(1.0f, L1 + eps_l1);
+  const float2 eps = f2(eps_log);
 #pragma unroll
-  for (int o = 0; o < C::NOCT; ++o) {
-    float v[8];
-    load_oct<C>(stage, (int)threadIdx.x, o, v);
+  for (int p = 0; p < NP; ++p) {
+    float2 t[8];
 #pragma unroll
     for (int k = 0; k < 8; ++k) {
-      const float p = fabsf(v[k]) * inv;
-      v[k] = p * lg2_poly(p + eps_log);
+      const float2 pk = f2(a[p][k].x * inv, a[p][k].y * inv);   // scalar: pk is added to below
+      t[k] = mul2(pk, lg2_poly2(add2(pk, eps)));
     }
-    part[o] = tree8(v);
+    // first tree level with scalar adds (its operands are packed products), the rest packed
+    const float2 s01 = f2(t[0].x + t[1].x, t[0].y + t[1].y), s23 = f2(t[2].x + t[3].x, t[2].y + t[3].y);
+    const float2 s45 = f2(t[4].x + t[5].x, t[4].y + t[5].y), s67 = f2(t[6].x + t[7].x, t[6].y + t[7].y);
+    const float2 s = add2(add2(s01, s23), add2(s45, s67));
+    part[2 * p] = s.x;
+    part[2 * p + 1] = s.y;
   }
   float S = tree<C::NOCT>(part);
   if constexpr (C::LPT == 2) S = S + __shfl_xor_sync(kFull, S, 1);
@@ -218,6 +323,94 @@ __device__ __forceinline__ void hadamard_scaled(float (&x)[C::EPT]) {
   constexpr float c = (C::G == 32) ? 0.17677669529663687f : (C::G == 64) ? 0.125f : 0.08838834764831845f;
 #pragma unroll
   for (int k = 0; k < C::EPT; ++k) x[k] = x[k] * c;
+}
+
+// The same butterfly on adjacent pairs p[i] = (x[2i], x[2i+1]): stride 1 works inside a pair, every
+// larger stride adds and subtracts whole pairs (a - b is formed as fma(b, -1, a), which is exact).
+template <int NPAIR>
+__device__ __forceinline__ void butterfly2(float2 (&p)[NPAIR]) {
+#pragma unroll
+  for (int i = 0; i < NPAIR; ++i) p[i] = make_float2(p[i].x + p[i].y, p[i].x - p[i].y);
+#pragma unroll
+  for (int h = 1; h < NPAIR; h *= 2)
+#pragma unroll
+    for (int i = 0; i < NPAIR; ++i)
+      if (!(i & h)) {
+        const float2 a = p[i], b = p[i + h];
+        p[i] = add2(a, b);
+        p[i + h] = fma2(b, f2(-1.0f), a);
+      }
+}
+
+// A row as adjacent pairs, widened to binary32.
+template <class C>
+__device__ __forceinline__ void load_row_pairs(const uint8_t *stage, int row, float2 (&p)[C::EPT / 2]) {
+#pragma unroll
+  for (int q = 0; q < C::CPR; ++q) {
+    const uint4 w = *reinterpret_cast<const uint4 *>(stage + (size_t)phys_chunk<C>(row, q) * 16);
+    if constexpr (C::BF16) {
+      const uint32_t u[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) bf2_add_f32(u[j], -0.0f, p[4 * q + j].x, p[4 * q + j].y);
+    } else {
+      p[2 * q] = make_float2(__uint_as_float(w.x), __uint_as_float(w.y));
+      p[2 * q + 1] = make_float2(__uint_as_float(w.z), __uint_as_float(w.w));
+    }
+  }
+}
+
+// First index whose magnitude equals m (the row's largest magnitude), scanning the row in shared memory.
+template <class C>
+__device__ __forceinline__ int row_first_index_of(const uint8_t *stage, int row, float m) {
+  int qhit = C::CPR - 1;
+  if constexpr (C::BF16) {
+    const uint32_t pat = __float_as_uint(m) >> 16;
+#pragma unroll
+    for (int q = C::CPR - 1; q >= 0; --q) {   // last assignment wins: the lowest chunk that holds the maximum
+      const uint4 w = *reinterpret_cast<const uint4 *>(stage + (size_t)phys_chunk<C>(row, q) * 16);
+      const uint32_t t = bf2_max_abs(bf2_max_abs(w.x, w.y), bf2_max_abs(w.z, w.w)) & 0x7fff7fffu;
+      qhit = (max(t & 0xffffu, t >> 16) == pat) ? q : qhit;
+    }
+    const uint4 w = *reinterpret_cast<const uint4 *>(stage + (size_t)phys_chunk<C>(row, qhit) * 16);
+    const uint32_t u[4] = {w.x, w.y, w.z, w.w};
+    int k = 7;
+#pragma unroll
+    for (int j = 3; j >= 0; --j) {
+      k = ((u[j] >> 16) & 0x7fffu) == pat ? 2 * j + 1 : k;
+      k = (u[j] & 0x7fffu) == pat ? 2 * j : k;
+    }
+    return qhit * 8 + k;
+  } else {
+#pragma unroll
+    for (int q = C::CPR - 1; q >= 0; --q) {
+      const float4 v = *reinterpret_cast<const float4 *>(stage + (size_t)phys_chunk<C>(row, q) * 16);
+      const float t = fmaxf(fmaxf(fabsf(v.x), fabsf(v.y)), fmaxf(fabsf(v.z), fabsf(v.w)));
+      qhit = (t == m) ? q : qhit;
+    }
+    const float4 v = *reinterpret_cast<const float4 *>(stage + (size_t)phys_chunk<C>(row, qhit) * 16);
+    int k = 3;
+    k = fabsf(v.z) == m ? 2 : k;
+    k = fabsf(v.y) == m ? 1 : k;
+    k = fabsf(v.x) == m ? 0 : k;
+    return qhit * 4 + k;
+  }
+}
+
+// Swap elements 0 and d of a row held in shared memory (the pivot swap P_d, its own inverse).
+template <class C, bool F32>
+__device__ __forceinline__ void row_swap_0_d(uint8_t *stage, int row, int d) {
+  constexpr int ES = F32 ? 4 : 2, EPC = 16 / ES;
+  uint8_t *p0 = stage + (size_t)phys_chunk<C>(row, 0) * 16;
+  uint8_t *pd = stage + (size_t)phys_chunk<C>(row, d / EPC) * 16 + (size_t)(d % EPC) * ES;
+  if constexpr (F32) {
+    const uint32_t a = *reinterpret_cast<uint32_t *>(p0), b = *reinterpret_cast<uint32_t *>(pd);
+    *reinterpret_cast<uint32_t *>(p0) = b;
+    *reinterpret_cast<uint32_t *>(pd) = a;
+  } else {
+    const uint16_t a = *reinterpret_cast<uint16_t *>(p0), b = *reinterpret_cast<uint16_t *>(pd);
+    *reinterpret_cast<uint16_t *>(p0) = b;
+    *reinterpret_cast<uint16_t *>(pd) = a;
+  }
 }
 
 // Little-endian bit stream of N codes of W bits into N*W/32 words (all indices static).
@@ -278,38 +471,6 @@ __device__ __forceinline__ ClassSort sort_by_class(int cls, uint8_t *s_perm, uin
   const int t = threadIdx.x;
   r.cls = (t >= base1) + (t >= base2) + (t >= base3);
   return r;
-}
-
-// ------------------------------------------------------------------------------------------
-// bf16 pairs handled in their packed form (sm_100a: packed bf16 min/max run on the ALU pipe, one
-// instruction per two elements; a bf16 operand can feed an fp32 add on the FMA pipe directly)
-// ------------------------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t bf2_max_abs(uint32_t a, uint32_t b) {   // magnitudes; sign bits are garbage
-  uint32_t d;
-  asm("max.xorsign.abs.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
-  return d;
-}
-__device__ __forceinline__ uint32_t bf2_min_abs(uint32_t a, uint32_t b) {
-  uint32_t d;
-  asm("min.xorsign.abs.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
-  return d;
-}
-__device__ __forceinline__ uint32_t bf2_max(uint32_t a, uint32_t b) {
-  uint32_t d;
-  asm("max.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
-  return d;
-}
-__device__ __forceinline__ uint32_t bf2_min(uint32_t a, uint32_t b) {
-  uint32_t d;
-  asm("min.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
-  return d;
-}
-// (lo + c, hi + c) in binary32 for the two bf16 halves of w: the widening is exact, so this equals
-// widening first and adding afterwards; with c = -0.0f it is the widening itself.
-__device__ __forceinline__ void bf2_add_f32(uint32_t w, float c, float &lo, float &hi) {
-  asm("{\n\t.reg .b16 l, h;\n\tmov.b32 {l, h}, %2;\n\tadd.rn.f32.bf16 %0, l, %3;\n\tadd.rn.f32.bf16 %1, h, %3;\n\t}"
-      : "=f"(lo), "=f"(hi)
-      : "r"(w), "f"(c));
 }
 
 // Largest and second-largest magnitude of a row (Eq. 3), no index.
@@ -382,18 +543,23 @@ __device__ __forceinline__ void pack_magic(F &&t, uint32_t *w) {
 // multiplying by s*2^-p inside the fused multiply-add gives the same real product q*s, so the result
 // is bit-identical to fma((float)q, s, z).
 template <int W, int N>
-__device__ __forceinline__ void unpack_dequant(const uint32_t *w, float s, float z, float (&x)[N]) {
+__device__ __forceinline__ void unpack_dequant(const uint32_t *w, float s, float z, float2 (&x)[N / 2]) {
   constexpr uint32_t M = (1u << W) - 1u;
 #pragma unroll
-  for (int k = 0; k < N; ++k) {
-    const int bit = k * W, j = bit >> 5, sh = bit & 31;
-    uint32_t src;
-    int p;
-    if (sh + W <= 23) { src = w[j]; p = sh; }
-    else if (sh + W <= 32) { src = w[j] >> 16; p = sh - 16; }
-    else { src = __funnelshift_r(w[j], w[j + 1], sh); p = 0; }
-    const float f = __uint_as_float((src & (M << p)) | 0x4B000000u) - 8388608.0f;
-    x[k] = __fmaf_rn(f, s * (1.0f / (float)(1u << p)), z);
+  for (int i = 0; i < N / 2; ++i) {
+    float f[2], sc[2];
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {
+      const int bit = (2 * i + e) * W, j = bit >> 5, sh = bit & 31;
+      uint32_t src;
+      int p;
+      if (sh + W <= 23) { src = w[j]; p = sh; }
+      else if (sh + W <= 32) { src = w[j] >> 16; p = sh - 16; }
+      else { src = __funnelshift_r(w[j], w[j + 1], sh); p = 0; }
+      f[e] = __uint_as_float((src & (M << p)) | 0x4B000000u);
+      sc[e] = s * (1.0f / (float)(1u << p));
+    }
+    x[i] = fma2(add2(f2(f[0], f[1]), f2(-8388608.0f)), f2(sc[0], sc[1]), f2(z));
   }
 }
 

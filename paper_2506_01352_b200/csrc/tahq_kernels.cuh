@@ -166,23 +166,6 @@ __global__ void __launch_bounds__(kThreads) stats_kernel(const Args a) {
 constexpr int kSelThreads = 1024;
 constexpr int kSortCap = 8192;   // candidates that are sorted in shared memory
 
-// Bitonic sort, descending, of n = 2^m keys in shared memory by the whole CTA.
-__device__ __forceinline__ void bitonic_desc(unsigned long long *s, uint32_t n) {
-  for (uint32_t k = 2; k <= n; k <<= 1) {
-    for (uint32_t j = k >> 1; j > 0; j >>= 1) {
-      for (uint32_t i = threadIdx.x; i < n; i += kSelThreads) {
-        const uint32_t p = i ^ j;
-        if (p > i) {
-          const unsigned long long x = s[i], y = s[p];
-          const bool desc = (i & k) == 0;
-          if (desc ? (x < y) : (x > y)) { s[i] = y; s[p] = x; }
-        }
-      }
-      __syncthreads();
-    }
-  }
-}
-
 // r-th largest (1-based) key of a sequence, radix select with 8 bits a pass.  get(i, key) returns
 // false for entries that do not take part.
 template <class Get>
@@ -228,6 +211,8 @@ __device__ __forceinline__ unsigned long long radix_select(uint64_t count, uint3
   return prefix;
 }
 
+constexpr int kSelSlice = 4 * kSelThreads;   // scores one CTA of select_kernel scans (four per thread, loaded at once)
+
 __global__ void __launch_bounds__(kSelThreads) select_kernel(const Args a) {
   extern __shared__ __align__(16) unsigned long long s_keys[];   // kSortCap keys
   __shared__ uint32_t s_warp[kSelThreads / 32];
@@ -237,21 +222,23 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const Args a) {
   const uint64_t ng = a.tiles_per_group;
   const float *sc = a.scores + g * ng;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-
-  auto sort_and_pick = [&](uint32_t n, uint32_t r) {   // keys [0, n) are in s_keys
-    uint32_t n2 = 2;
-    while (n2 < n) n2 <<= 1;
-    for (uint32_t i = n + threadIdx.x; i < n2; i += kSelThreads) s_keys[i] = 0;   // below every real key
-    __syncthreads();
-    bitonic_desc(s_keys, n2);
-    if (threadIdx.x == 0) a.theta[g] = s_keys[r - 1];
-  };
+  auto from_smem = [&](uint64_t i, unsigned long long &key) { key = s_keys[i]; return true; };
 
   if (a.direct) {   // small group: rank all of its tiles here (one CTA per group)
     for (uint32_t i = threadIdx.x; i < (uint32_t)ng; i += kSelThreads) s_keys[i] = rank_key(sc[i], i);
     __syncthreads();
-    sort_and_pick((uint32_t)ng, (uint32_t)a.k_hi);
+    const unsigned long long t = radix_select(ng, (uint32_t)a.k_hi, from_smem);
+    if (threadIdx.x == 0) a.theta[g] = t;
     return;
+  }
+
+  // this CTA's slice of the group's scores, in flight while the threshold bin is being found
+  const uint64_t lo = (blockIdx.x % a.cpg) * (uint64_t)kSelSlice;
+  float sv[4];
+#pragma unroll
+  for (int u = 0; u < 4; ++u) {
+    const uint64_t i = lo + (uint64_t)u * kSelThreads + threadIdx.x;
+    sv[u] = i < ng ? __ldg(sc + i) : 0.0f;
   }
 
   // ---- A: the bin that holds the k_hi-th ranked tile (every CTA of the group finds it for itself)
@@ -260,8 +247,7 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const Args a) {
   uint32_t hb[BPT], mine = 0;
 #pragma unroll
   for (int j = 0; j < BPT; ++j) { hb[j] = gh[threadIdx.x * BPT + j]; mine += hb[j]; }
-  // suffix sums: tiles in bins above this thread's bins
-  uint32_t incl = mine;
+  uint32_t incl = mine;   // suffix sums: tiles in bins above this thread's bins
 #pragma unroll
   for (int o = 1; o < 32; o *= 2) {
     const uint32_t v = __shfl_down_sync(kFull, incl, o);
@@ -282,22 +268,18 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const Args a) {
   __syncthreads();
   const uint32_t B = s_sel[0], r = s_sel[1];
 
-  // ---- B: this CTA's slice of the group: candidates of bin B go to the group's list
-  const uint64_t j = blockIdx.x % a.cpg;
-  const uint64_t slice = (ng + a.cpg - 1) / a.cpg;
-  const uint64_t lo = j * slice < ng ? j * slice : ng;
-  const uint64_t hi = lo + slice < ng ? lo + slice : ng;
-  for (uint64_t i0 = lo; i0 < hi; i0 += kSelThreads) {   // whole warps stay in the loop: one atomic per warp
-    const uint64_t i = i0 + threadIdx.x;
-    const float s = i < hi ? sc[i] : 0.0f;
-    const bool take = i < hi && score_bin(s) == B;
+  // ---- B: candidates of bin B go to the group's list (one atomic per warp)
+#pragma unroll
+  for (int u = 0; u < 4; ++u) {
+    const uint64_t i = lo + (uint64_t)u * kSelThreads + threadIdx.x;
+    const bool take = i < ng && score_bin(sv[u]) == B;
     const unsigned m = __ballot_sync(kFull, take);
     if (m) {
       uint32_t base = 0;
       if (lane == 0) base = atomicAdd(&a.ncand[g], (uint32_t)__popc(m));
       base = __shfl_sync(kFull, base, 0);
       const uint32_t slot = base + __popc(m & ((1u << lane) - 1u));
-      if (take && slot < a.cand_cap) a.cand[g * a.cand_cap + slot] = rank_key(s, (uint32_t)i);
+      if (take && slot < a.cand_cap) a.cand[g * a.cand_cap + slot] = rank_key(sv[u], (uint32_t)i);
     }
   }
 
@@ -310,24 +292,24 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const Args a) {
   __threadfence();
   const uint32_t n = gh[B];
   const unsigned long long *cand = a.cand + g * a.cand_cap;
+  unsigned long long t;
   if (n <= a.cand_cap && n <= (uint32_t)kSortCap) {
     for (uint32_t i = threadIdx.x; i < n; i += kSelThreads) s_keys[i] = __ldcg(cand + i);
     __syncthreads();
-    sort_and_pick(n, r);
+    t = radix_select(n, r, from_smem);
   } else if (n <= a.cand_cap) {
-    const unsigned long long t = radix_select(n, r, [&](uint64_t i, unsigned long long &key) {
+    t = radix_select(n, r, [&](uint64_t i, unsigned long long &key) {
       key = __ldcg(cand + i);
       return true;
     });
-    if (threadIdx.x == 0) a.theta[g] = t;
   } else {   // more candidates than the list holds: take them from the scores
-    const unsigned long long t = radix_select(ng, r, [&](uint64_t i, unsigned long long &key) {
+    t = radix_select(ng, r, [&](uint64_t i, unsigned long long &key) {
       const float s = sc[i];
       key = rank_key(s, (uint32_t)i);
       return score_bin(s) == B;
     });
-    if (threadIdx.x == 0) a.theta[g] = t;
   }
+  if (threadIdx.x == 0) a.theta[g] = t;
 }
 
 // Is tile `tile` one of the k_hi highest-ranked tiles of its group?
@@ -475,43 +457,67 @@ __device__ __forceinline__ Quantiser make_quantiser(float mn, float mx, uint32_t
   return q;
 }
 
-// t[k] = clamp((x[k] - z) * inv_s, 0, qmax) + 1.5*2^23.  The clamp is skipped when the whole warp's
-// rows provably stay inside [-0.5, qmax + 0.5) (the two operations are monotone in x), where it
-// cannot change the rounded code.
+// t[k] = 1.5*2^23 + round(clamp((x[k] - z) * inv_s, 0, qmax)): the difference is a binary32
+// subtraction, and the fused multiply-add rounds the exact product once, straight to an integer
+// (ties to even).  Clamping the sum to [1.5*2^23, 1.5*2^23 + qmax] equals clamping the product; it
+// is skipped when the whole warp's rows provably stay inside [-0.5, qmax + 0.5) (subtraction and
+// product are monotone in x), where it cannot change the code.
 template <int N>
 __device__ __forceinline__ void quantise_row(float (&x)[N], float mn, float mx, const Quantiser &q) {
   const float ymin = (mn - q.z) * q.inv_s, ymax = (mx - q.z) * q.inv_s;
-  const bool safe = ymin >= -0.5f && ymax < q.qmax + 0.5f;
+  const bool safe = ymin >= -0.4999f && ymax < q.qmax + 0.4999f;
   if (__all_sync(__activemask(), safe)) {
 #pragma unroll
-    for (int k = 0; k < N; ++k) x[k] = (x[k] - q.z) * q.inv_s + kMagic;
+    for (int k = 0; k < N; ++k) x[k] = __fmaf_rn(x[k] - q.z, q.inv_s, kMagic);
   } else {
 #pragma unroll
-    for (int k = 0; k < N; ++k) x[k] = fminf(fmaxf((x[k] - q.z) * q.inv_s, 0.0f), q.qmax) + kMagic;
+    for (int k = 0; k < N; ++k)
+      x[k] = fminf(fmaxf(__fmaf_rn(x[k] - q.z, q.inv_s, kMagic), kMagic), kMagic + q.qmax);
   }
 }
 
-// t(k) must return q_k + 1.5*2^23 for a compile-time k; the codes leave as N*bits/32 words.
-template <int N, class F>
-__device__ __forceinline__ void pack_row(F &&t, uint32_t bits, uint32_t *dst) {
-  uint32_t w[N / 4];
-  switch (bits) {
-    case 2: pack_magic<2, N>(t, w); break;
-    case 3: pack_magic<3, N>(t, w); break;
-    case 4: pack_magic<4, N>(t, w); break;
-    case 5: pack_magic<5, N>(t, w); break;
-    case 6: pack_magic<6, N>(t, w); break;
-    case 7: pack_magic<7, N>(t, w); break;
-    default: pack_magic<8, N>(t, w); break;
-  }
-  if constexpr (N == 64) {   // 64-wide rows start on 8-byte boundaries of the staging buffer
+// t(k) must return q_k + 1.5*2^23 for a compile-time k; the row's N*bits/32 words go straight to
+// the payload (rows of 64 codes start on 8-byte boundaries).
+template <int W, int N, class F>
+__device__ __forceinline__ void pack_store(F &&t, uint32_t *dst) {
+  uint32_t w[N * W / 32];
+  pack_magic<W, N>(t, w);
+  if constexpr (N == 64) {
 #pragma unroll
-    for (int j = 0; j < N / 8; ++j)
-      if (j < (int)(N * bits / 64)) reinterpret_cast<uint2 *>(dst)[j] = make_uint2(w[2 * j], w[2 * j + 1]);
+    for (int j = 0; j < W; ++j) reinterpret_cast<uint2 *>(dst)[j] = make_uint2(w[2 * j], w[2 * j + 1]);
   } else {
 #pragma unroll
-    for (int j = 0; j < N / 4; ++j)
-      if (j < (int)(N * bits / 32)) dst[j] = w[j];
+    for (int j = 0; j < N * W / 32; ++j) dst[j] = w[j];
+  }
+}
+template <int N, class F>
+__device__ __forceinline__ void pack_row(F &&t, uint32_t bits, uint32_t *dst) {
+  switch (bits) {
+    case 2: pack_store<2, N>(t, dst); break;
+    case 3: pack_store<3, N>(t, dst); break;
+    case 4: pack_store<4, N>(t, dst); break;
+    case 5: pack_store<5, N>(t, dst); break;
+    case 6: pack_store<6, N>(t, dst); break;
+    case 7: pack_store<7, N>(t, dst); break;
+    default: pack_store<8, N>(t, dst); break;
+  }
+}
+
+// The same for a row held as adjacent pairs (two elements per instruction).
+template <int NPAIR>
+__device__ __forceinline__ void quantise_pairs(float2 (&p)[NPAIR], float mn, float mx, const Quantiser &q) {
+  const float ymin = (mn - q.z) * q.inv_s, ymax = (mx - q.z) * q.inv_s;
+  const bool safe = ymin >= -0.4999f && ymax < q.qmax + 0.4999f;
+  const float2 nz = f2(-q.z), is = f2(q.inv_s), mg = f2(kMagic);
+  if (__all_sync(__activemask(), safe)) {
+#pragma unroll
+    for (int i = 0; i < NPAIR; ++i) p[i] = fma2(add2(p[i], nz), is, mg);
+  } else {
+#pragma unroll
+    for (int i = 0; i < NPAIR; ++i) {
+      const float2 t = fma2(add2(p[i], nz), is, mg);
+      p[i] = f2(fminf(fmaxf(t.x, kMagic), kMagic + q.qmax), fminf(fmaxf(t.y, kMagic), kMagic + q.qmax));
+    }
   }
 }
 
@@ -537,20 +543,22 @@ __device__ __forceinline__ Quantiser encode_raw_bf16_row(const uint8_t *stage, i
   const float mx = fmaxf(__uint_as_float(hi0 << 16), __uint_as_float(hi0 & 0xffff0000u));
   const Quantiser q = make_quantiser(mn, mx, bits);
   const float ymin = (mn - q.z) * q.inv_s, ymax = (mx - q.z) * q.inv_s;
-  const bool safe = ymin >= -0.5f && ymax < q.qmax + 0.5f;
+  const bool safe = ymin >= -0.4999f && ymax < q.qmax + 0.4999f;
   const float nz = -q.z;   // x + (-z) is x - z
+  const float2 is = f2(q.inv_s), mg = f2(kMagic);
   if (__all_sync(__activemask(), safe)) {
     auto t = [&](int k) {
-      float a, b;
-      bf2_add_f32(w[k >> 1], nz, a, b);
-      return ((k & 1) ? b : a) * q.inv_s + kMagic;
+      float2 d;
+      bf2_add_f32(w[k >> 1], nz, d.x, d.y);
+      d = fma2(d, is, mg);
+      return (k & 1) ? d.y : d.x;
     };
     if (store) pack_row<C::EPT>(t, bits, dst);
   } else {
     auto t = [&](int k) {
       float a, b;
       bf2_add_f32(w[k >> 1], nz, a, b);
-      return fminf(fmaxf(((k & 1) ? b : a) * q.inv_s, 0.0f), q.qmax) + kMagic;
+      return fminf(fmaxf(__fmaf_rn((k & 1) ? b : a, q.inv_s, kMagic), kMagic), kMagic + q.qmax);
     };
     if (store) pack_row<C::EPT>(t, bits, dst);
   }
@@ -560,7 +568,6 @@ __device__ __forceinline__ Quantiser encode_raw_bf16_row(const uint8_t *stage, i
 template <class C, int NST>
 __global__ void __launch_bounds__(kThreads, 2) quant_pack_kernel(const Args a) {
   extern __shared__ __align__(128) uint8_t smem[];
-  uint32_t *out = reinterpret_cast<uint32_t *>(smem + (size_t)NST * C::STAGE_BYTES);
   __shared__ uint8_t s_perm[kThreads];
   __shared__ uint2 s_cnt[kThreads / 32];
   __shared__ uint16_t s_rowoff[kThreads];
@@ -606,7 +613,6 @@ __global__ void __launch_bounds__(kThreads, 2) quant_pack_kernel(const Args a) {
     const uint32_t nvalid = left < (uint64_t)C::TPC ? (uint32_t)left : (uint32_t)C::TPC;
     const uint32_t own = threadIdx.x / C::LPT;   // tile of the chunk this thread looks at first
     const bool hi1 = a.mixed && own < nvalid && cur.is_hi(a, tile0 + own, own);
-    uint32_t chunk_bytes;
     const uint64_t goff = (uint64_t)(C::G / 8) * ((uint64_t)a.lo * tile0 + hi_run);
 
     if constexpr (C::LPT == 1) {
@@ -621,7 +627,6 @@ __global__ void __launch_bounds__(kThreads, 2) quant_pack_kernel(const Args a) {
         s_a1[threadIdx.x] = a1;
         if ((threadIdx.x & 31) == 0) bitmap[tile0 / 32 + (threadIdx.x >> 5)] = r.hi_ballot;
       });
-      chunk_bytes = (C::G / 8) * (a.lo * nvalid + rg.total_hi);
       hi_run += rg.total_hi;
       // ---- phase 2: this thread now owns tile `src` of the chunk
       const int src = rg.src;
@@ -629,41 +634,37 @@ __global__ void __launch_bounds__(kThreads, 2) quant_pack_kernel(const Args a) {
       const uint32_t b = a.lo + (rg.cls & 1);
       const uint64_t tile = tile0 + src;
       const bool live = (uint32_t)src < nvalid;
-      uint32_t *dst = out + s_rowoff[src] / 4;
+      uint32_t *dst = reinterpret_cast<uint32_t *>(a.packed + a.off_payload + goff + s_rowoff[src]);
       if (C::BF16 && !flag) {
         const Quantiser q = encode_raw_bf16_row<C>(stage, src, b, dst, live);
         if (live) { sz32[tile] = q.sz; pivot[tile] = 0; }
       } else {
-        float x[C::EPT];
-#pragma unroll
-        for (int o = 0; o < C::NOCT; ++o) {
-          float v[8];
-          load_oct<C>(stage, src, o, v);
-#pragma unroll
-          for (int k = 0; k < 8; ++k) x[8 * o + k] = v[k];
-        }
         int d = 0;
-        if (flag) {   // Eq. 4: pivot swap + Hadamard
-          const float m = s_a1[src];
-#pragma unroll
-          for (int k = C::EPT - 1; k >= 0; --k) d = (fabsf(x[k]) == m) ? k : d;   // first index of the maximum
-          const float xd = load_elem<C>(stage, src, d), x0 = x[0];
-#pragma unroll
-          for (int k = 1; k < C::EPT; ++k) x[k] = (k == d) ? x0 : x[k];
-          x[0] = xd;
-          butterfly<C::EPT>(x);
-#pragma unroll
-          for (int k = 0; k < C::EPT; ++k) x[k] = x[k] * hadamard_scale<C>();
+        if (flag) {   // Eq. 4: the pivot swap P_d, done in place in shared memory before the row is loaded
+          d = row_first_index_of<C>(stage, src, s_a1[src]);
+          row_swap_0_d<C, !C::BF16>(const_cast<uint8_t *>(stage), src, d);
+          asm volatile("" ::: "memory");
         }
-        float mn = x[0], mx = x[0];
+        float2 p[C::EPT / 2];
+        load_row_pairs<C>(stage, src, p);
+        if (flag) {   // Eq. 4: (1/sqrt G) H_G
+          butterfly2<C::EPT / 2>(p);
 #pragma unroll
-        for (int k = 1; k < C::EPT; ++k) { mn = fminf(mn, x[k]); mx = fmaxf(mx, x[k]); }
+          for (int i = 0; i < C::EPT / 2; ++i)   // scalar products: they are added to right after
+            p[i] = f2(p[i].x * hadamard_scale<C>(), p[i].y * hadamard_scale<C>());
+        }
+        float mn = fminf(p[0].x, p[0].y), mx = fmaxf(p[0].x, p[0].y);
+#pragma unroll
+        for (int i = 1; i < C::EPT / 2; ++i) {
+          mn = fminf(mn, fminf(p[i].x, p[i].y));
+          mx = fmaxf(mx, fmaxf(p[i].x, p[i].y));
+        }
         const Quantiser q = make_quantiser(mn, mx, b);
-        quantise_row<C::EPT>(x, mn, mx, q);
+        quantise_pairs<C::EPT / 2>(p, mn, mx, q);
         if (live) {
           sz32[tile] = q.sz;
           pivot[tile] = flag ? (uint8_t)(0x80 | d) : (uint8_t)0;
-          pack_row<C::EPT>([&](int k) { return x[k]; }, b, dst);
+          pack_row<C::EPT>([&](int k) { return (k & 1) ? p[k >> 1].y : p[k >> 1].x; }, b, dst);
         }
       }
     } else {
@@ -674,7 +675,6 @@ __global__ void __launch_bounds__(kThreads, 2) quant_pack_kernel(const Args a) {
       pair_scan(hi1, reinterpret_cast<uint32_t *>(s_cnt), hi_before, total_hi, tiles16);
       if ((threadIdx.x & 31) == 0)
         reinterpret_cast<uint16_t *>(bitmap)[tile0 / 16 + (threadIdx.x >> 5)] = (uint16_t)tiles16;
-      chunk_bytes = (C::G / 8) * (a.lo * nvalid + total_hi);
       hi_run += total_hi;
       const uint32_t b = a.lo + (hi1 ? 1u : 0u);
       const uint32_t row_off = (C::G / 8) * (a.lo * own + hi_before) + half * (C::EPT / 8) * b;
@@ -740,20 +740,11 @@ __global__ void __launch_bounds__(kThreads, 2) quant_pack_kernel(const Args a) {
           sz32[tile] = q.sz;
           pivot[tile] = flag ? (uint8_t)(0x80 | d) : (uint8_t)0;
         }
-        pack_row<C::EPT>([&](int k) { return x[k]; }, b, out + row_off / 4);
+        pack_row<C::EPT>([&](int k) { return x[k]; }, b,
+                         reinterpret_cast<uint32_t *>(a.packed + a.off_payload + goff + row_off));
       }
     }
     cur.advance(a, C::TPC);
-    __syncthreads();
-    // the chunk's codes leave with coalesced stores (payload offsets are multiples of G/8 bytes)
-    if constexpr (C::G >= 64) {
-      uint2 *gdst = reinterpret_cast<uint2 *>(a.packed + a.off_payload + goff);
-      const uint2 *s2 = reinterpret_cast<const uint2 *>(out);
-      for (uint32_t i = threadIdx.x; i < chunk_bytes / 8; i += kThreads) gdst[i] = s2[i];
-    } else {
-      uint32_t *gdst = reinterpret_cast<uint32_t *>(a.packed + a.off_payload + goff);
-      for (uint32_t i = threadIdx.x; i < chunk_bytes / 4; i += kThreads) gdst[i] = out[i];
-    }
   });
 }
 
@@ -762,7 +753,7 @@ __global__ void __launch_bounds__(kThreads, 2) quant_pack_kernel(const Args a) {
 // ------------------------------------------------------------------------------------------
 
 template <int N>
-__device__ __forceinline__ void load_dequant(const uint32_t *src, uint32_t bits, float s, float z, float (&x)[N]) {
+__device__ __forceinline__ void load_dequant(const uint32_t *src, uint32_t bits, float s, float z, float2 (&x)[N / 2]) {
   uint32_t w[N / 4];
   if constexpr (N == 64) {   // 64-wide rows start on 8-byte boundaries
 #pragma unroll
@@ -786,16 +777,17 @@ __device__ __forceinline__ void load_dequant(const uint32_t *src, uint32_t bits,
   }
 }
 
-// Store a register row into the swizzled output stage (narrowing to bf16 with round-to-nearest-even).
+// Store a row held as adjacent pairs into the swizzled output stage (narrowing to bf16 with
+// round-to-nearest-even).
 template <class C>
-__device__ __forceinline__ void stage_row(uint8_t *stage, int row, const float (&x)[C::EPT]) {
+__device__ __forceinline__ void stage_row(uint8_t *stage, int row, const float2 (&p)[C::EPT / 2]) {
   if constexpr (C::BF16) {
 #pragma unroll
     for (int q = 0; q < C::CPR; ++q) {
       uint32_t u[4];
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
-        const __nv_bfloat162 h2 = __floats2bfloat162_rn(x[8 * q + 2 * j], x[8 * q + 2 * j + 1]);
+        const __nv_bfloat162 h2 = __floats2bfloat162_rn(p[4 * q + j].x, p[4 * q + j].y);
         u[j] = *reinterpret_cast<const uint32_t *>(&h2);
       }
       *reinterpret_cast<uint4 *>(stage + (size_t)phys_chunk<C>(row, q) * 16) = make_uint4(u[0], u[1], u[2], u[3]);
@@ -804,7 +796,7 @@ __device__ __forceinline__ void stage_row(uint8_t *stage, int row, const float (
 #pragma unroll
     for (int q = 0; q < C::CPR; ++q)
       *reinterpret_cast<float4 *>(stage + (size_t)phys_chunk<C>(row, q) * 16) =
-          make_float4(x[4 * q], x[4 * q + 1], x[4 * q + 2], x[4 * q + 3]);
+          make_float4(p[2 * q].x, p[2 * q].y, p[2 * q + 1].x, p[2 * q + 1].y);
   }
 }
 
@@ -861,7 +853,7 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const Args a) {
     const uint32_t own = threadIdx.x / C::LPT;
     const uint64_t goff = (uint64_t)(C::G / 8) * ((uint64_t)a.lo * tile0 + hi_run);
     const uint8_t *pay = a.packed + a.off_payload + goff;
-    float x[C::EPT];
+    float2 x[C::EPT / 2];
     bool hi1 = false;
     if (a.mixed && own < nvalid) hi1 = (__ldg(bitmap + (tile0 + own) / 32) >> ((tile0 + own) & 31)) & 1u;
     uint32_t chunk_bytes;
@@ -888,22 +880,18 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const Args a) {
         load_dequant<C::EPT>(reinterpret_cast<const uint32_t *>(pay + s_rowoff[src]), b, s, z, x);
       } else {
 #pragma unroll
-        for (int k = 0; k < C::EPT; ++k) x[k] = 0.0f;
+        for (int i = 0; i < C::EPT / 2; ++i) x[i] = f2(0.0f);
       }
-      if (flag) {
-        const int d = s_pv[src] & 0x7f;
-        butterfly<C::EPT>(x);
+      if (flag) {   // (1/sqrt G) H_G^T = the same butterfly
+        butterfly2<C::EPT / 2>(x);
 #pragma unroll
-        for (int k = 0; k < C::EPT; ++k) x[k] = x[k] * hadamard_scale<C>();
-        float xd = x[0];   // un-swap coordinates 0 and d
-#pragma unroll
-        for (int k = 1; k < C::EPT; ++k) xd = (k == d) ? x[k] : xd;
-        const float x0 = x[0];
-#pragma unroll
-        for (int k = 1; k < C::EPT; ++k) x[k] = (k == d) ? x0 : x[k];
-        x[0] = xd;
+        for (int i = 0; i < C::EPT / 2; ++i) x[i] = mul2(x[i], f2(hadamard_scale<C>()));
       }
       stage_row<C>(smem, src, x);
+      if (flag) {   // un-swap coordinates 0 and d in the staged row
+        asm volatile("" ::: "memory");
+        row_swap_0_d<C, !C::BF16>(smem, src, s_pv[src] & 0x7f);
+      }
     } else {
       const int half = threadIdx.x & 1;
       const uint64_t tile = tile0 + own;
@@ -923,31 +911,34 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const Args a) {
         load_dequant<C::EPT>(reinterpret_cast<const uint32_t *>(pay + row_off), b, s, z, x);
       } else {
 #pragma unroll
-        for (int k = 0; k < C::EPT; ++k) x[k] = 0.0f;
+        for (int i = 0; i < C::EPT / 2; ++i) x[i] = f2(0.0f);
       }
       const bool flag = (pv & 0x80u) != 0;
       const unsigned fm = __ballot_sync(kFull, flag);
       if (flag) {
         const int d = pv & 0x7f;
-        butterfly<C::EPT>(x);
+        butterfly2<C::EPT / 2>(x);
 #pragma unroll
-        for (int k = 0; k < C::EPT; ++k) {
-          const float p = __shfl_xor_sync(fm, x[k], 1);
-          x[k] = half ? (p - x[k]) : (x[k] + p);
+        for (int i = 0; i < C::EPT / 2; ++i) {   // last stage: across the two lanes of the tile
+          const float px = __shfl_xor_sync(fm, x[i].x, 1), py = __shfl_xor_sync(fm, x[i].y, 1);
+          x[i] = half ? make_float2(px - x[i].x, py - x[i].y) : make_float2(x[i].x + px, x[i].y + py);
         }
 #pragma unroll
-        for (int k = 0; k < C::EPT; ++k) x[k] = x[k] * hadamard_scale<C>();
+        for (int i = 0; i < C::EPT / 2; ++i) x[i] = mul2(x[i], f2(hadamard_scale<C>()));
         const int lane = threadIdx.x & 31, owner = d / C::EPT, dl = d % C::EPT;
-        float mine = x[0];
+        float mine = x[0].x;   // un-swap coordinates 0 and d (d may sit in the other lane)
 #pragma unroll
-        for (int k = 1; k < C::EPT; ++k) mine = (k == dl) ? x[k] : mine;
-        const float x0 = __shfl_sync(fm, x[0], lane & ~1);
+        for (int k = 1; k < C::EPT; ++k) mine = (k == dl) ? ((k & 1) ? x[k >> 1].y : x[k >> 1].x) : mine;
+        const float x0 = __shfl_sync(fm, x[0].x, lane & ~1);
         const float xd = __shfl_sync(fm, mine, (lane & ~1) + owner);
         if (half == owner) {
 #pragma unroll
-          for (int k = 0; k < C::EPT; ++k) x[k] = (k == dl) ? x0 : x[k];
+          for (int k = 0; k < C::EPT; ++k) {
+            if (k & 1) x[k >> 1].y = (k == dl) ? x0 : x[k >> 1].y;
+            else x[k >> 1].x = (k == dl) ? x0 : x[k >> 1].x;
+          }
         }
-        if (half == 0) x[0] = xd;
+        if (half == 0) x[0].x = xd;
       }
       stage_row<C>(smem, (int)threadIdx.x, x);
     }
