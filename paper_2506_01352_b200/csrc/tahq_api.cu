@@ -67,6 +67,7 @@ static tahq_status make_plan(const tahq_params *p, Plan *pl) {
   L.tiles_per_group = S * M;
   L.n_groups = p->tokens / S;
   if (L.tiles_per_group >= (1ull << 32) || L.n_tiles >= (1ull << 36)) return TAHQ_ERR_INVALID_ARG;
+  if (L.n_tiles > (uint64_t)kMaxGrid * kChunkCap * 128) return TAHQ_ERR_UNSUPPORTED;   // one call: up to 2^28 tiles
   pl->f = beta % 1000;
   L.lo_bits = beta / 1000;
   L.hi_bits = pl->f ? L.lo_bits + 1 : L.lo_bits;
@@ -225,11 +226,14 @@ static tahq_status decode_t(const Plan &pl, const Args &a, cudaStream_t st) {
   if (!dev_info(&d)) return TAHQ_ERR_CUDA;
   const uint64_t n_chunks = (a.n_tiles + C::TPC - 1) / C::TPC;
   static std::atomic<int> occ_dec[64];
-  const int smem = C::STAGE_BYTES;
+  const int smem = DecSmem<C>::TOTAL;
   const int occ = prepare(decode_kernel<C>, smem, d, occ_dec);
   if (!occ) return TAHQ_ERR_CUDA;
   (void)pl;
-  TAHQ_LAUNCH("decode", st, decode_kernel<C><<<persistent_grid(n_chunks, d, occ), kThreads, smem, st>>>(a));
+  unsigned grid = persistent_grid(n_chunks, d, occ);
+  const uint64_t need = (n_chunks + kChunkCap - 1) / kChunkCap;   // a CTA keeps its chunks' bit map in shared memory
+  if (grid < need) grid = (unsigned)need;
+  TAHQ_LAUNCH("decode", st, decode_kernel<C><<<grid, kThreads, smem, st>>>(a));
   return cudaGetLastError() == cudaSuccess ? TAHQ_OK : TAHQ_ERR_CUDA;
 }
 

@@ -62,6 +62,39 @@ __device__ __forceinline__ void cp_async_wait() {
   asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory");
 }
 
+// ------------------------------------------------------------------------------------------
+// Bulk asynchronous copies (TMA, untiled) completing on an mbarrier: one thread moves a whole
+// contiguous slice; addresses and sizes are multiples of 16 bytes.  Every wait is bounded.
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ unsigned smem_u32(const void *p) { return (unsigned)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(unsigned long long *bar, unsigned count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_init_fence() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+__device__ __forceinline__ void mbar_expect_tx(unsigned long long *bar, unsigned bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void bulk_copy_g2s(void *dst, const void *src, unsigned bytes, unsigned long long *bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                   smem_u32(dst)),
+               "l"(src), "r"(bytes), "r"(smem_u32(bar))
+               : "memory");
+}
+__device__ __forceinline__ void fence_async_proxy() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+// true when the phase with the given parity has completed; gives up after a bounded number of polls
+__device__ __forceinline__ bool mbar_wait(unsigned long long *bar, unsigned parity) {
+  for (unsigned spins = 0; spins < (1u << 22); ++spins) {
+    unsigned ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    if (ok) return true;
+  }
+  return false;
+}
+
 // Copy the rows of chunk `c` (tiles [c*TPC, (c+1)*TPC), clipped to n_tiles) into a swizzled stage.
 // Rows past the end of the tensor are zero-filled.
 template <class C>
@@ -543,23 +576,22 @@ __device__ __forceinline__ void pack_magic(F &&t, uint32_t *w) {
 // multiplying by s*2^-p inside the fused multiply-add gives the same real product q*s, so the result
 // is bit-identical to fma((float)q, s, z).
 template <int W, int N>
-__device__ __forceinline__ void unpack_dequant(const uint32_t *w, float s, float z, float2 (&x)[N / 2]) {
+__device__ __forceinline__ void unpack_dequant(const uint32_t *w, float s, float z, float (&x)[N]) {
   constexpr uint32_t M = (1u << W) - 1u;
+  uint32_t two23;   // 2^23 as a bit pattern, kept in a register so that (src & mask) | 2^23 is one instruction
+  asm volatile("mov.u32 %0, 0x4B000000;" : "=r"(two23));
 #pragma unroll
-  for (int i = 0; i < N / 2; ++i) {
-    float f[2], sc[2];
-#pragma unroll
-    for (int e = 0; e < 2; ++e) {
-      const int bit = (2 * i + e) * W, j = bit >> 5, sh = bit & 31;
-      uint32_t src;
-      int p;
-      if (sh + W <= 23) { src = w[j]; p = sh; }
-      else if (sh + W <= 32) { src = w[j] >> 16; p = sh - 16; }
-      else { src = __funnelshift_r(w[j], w[j + 1], sh); p = 0; }
-      f[e] = __uint_as_float((src & (M << p)) | 0x4B000000u);
-      sc[e] = s * (1.0f / (float)(1u << p));
-    }
-    x[i] = fma2(add2(f2(f[0], f[1]), f2(-8388608.0f)), f2(sc[0], sc[1]), f2(z));
+  for (int k = 0; k < N; ++k) {
+    const int bit = k * W, j = bit >> 5, sh = bit & 31;
+    uint32_t src;
+    int p;
+    if (sh + W <= 23) { src = w[j]; p = sh; }
+    else if (sh + W <= 32) { src = w[j] >> 16; p = sh - 16; }
+    else { src = __funnelshift_r(w[j], w[j + 1], sh); p = 0; }
+    uint32_t m;
+    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(m) : "r"(src), "r"(M << p), "r"(two23));   // (src & mask) | 2^23
+    const float f = __uint_as_float(m) - 8388608.0f;   // q * 2^p, exact
+    x[k] = __fmaf_rn(f, s * (1.0f / (float)(1u << p)), z);
   }
 }
 

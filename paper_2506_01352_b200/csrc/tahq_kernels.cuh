@@ -752,68 +752,89 @@ __global__ void __launch_bounds__(kThreads, 2) quant_pack_kernel(const Args a) {
 // Decode
 // ------------------------------------------------------------------------------------------
 
-template <int N>
-__device__ __forceinline__ void load_dequant(const uint32_t *src, uint32_t bits, float s, float z, float2 (&x)[N / 2]) {
-  uint32_t w[N / 4];
+// Bit stream (in shared memory) -> dequantised row z + q*s.
+template <int W, int N>
+__device__ __forceinline__ void load_dequant_w(const uint8_t *src, float s, float z, float (&x)[N]) {
+  uint32_t w[N * W / 32];
   if constexpr (N == 64) {   // 64-wide rows start on 8-byte boundaries
 #pragma unroll
-    for (int j = 0; j < N / 8; ++j) {
-      uint2 v = make_uint2(0u, 0u);
-      if (j < (int)(N * bits / 64)) v = __ldg(reinterpret_cast<const uint2 *>(src) + j);
+    for (int j = 0; j < W; ++j) {
+      const uint2 v = reinterpret_cast<const uint2 *>(src)[j];
       w[2 * j] = v.x; w[2 * j + 1] = v.y;
     }
   } else {
 #pragma unroll
-    for (int j = 0; j < N / 4; ++j) w[j] = (j < (int)(N * bits / 32)) ? __ldg(src + j) : 0u;
+    for (int j = 0; j < N * W / 32; ++j) w[j] = reinterpret_cast<const uint32_t *>(src)[j];
   }
+  unpack_dequant<W, N>(w, s, z, x);
+}
+template <int N>
+__device__ __forceinline__ void load_dequant(const uint8_t *src, uint32_t bits, float s, float z, float (&x)[N]) {
   switch (bits) {
-    case 2: unpack_dequant<2, N>(w, s, z, x); break;
-    case 3: unpack_dequant<3, N>(w, s, z, x); break;
-    case 4: unpack_dequant<4, N>(w, s, z, x); break;
-    case 5: unpack_dequant<5, N>(w, s, z, x); break;
-    case 6: unpack_dequant<6, N>(w, s, z, x); break;
-    case 7: unpack_dequant<7, N>(w, s, z, x); break;
-    default: unpack_dequant<8, N>(w, s, z, x); break;
+    case 2: load_dequant_w<2, N>(src, s, z, x); break;
+    case 3: load_dequant_w<3, N>(src, s, z, x); break;
+    case 4: load_dequant_w<4, N>(src, s, z, x); break;
+    case 5: load_dequant_w<5, N>(src, s, z, x); break;
+    case 6: load_dequant_w<6, N>(src, s, z, x); break;
+    case 7: load_dequant_w<7, N>(src, s, z, x); break;
+    default: load_dequant_w<8, N>(src, s, z, x); break;
   }
 }
 
-// Store a row held as adjacent pairs into the swizzled output stage (narrowing to bf16 with
-// round-to-nearest-even).
+// A register row -> 16-byte pieces in the element type of the tensor (bf16: round-to-nearest-even).
 template <class C>
-__device__ __forceinline__ void stage_row(uint8_t *stage, int row, const float2 (&p)[C::EPT / 2]) {
+__device__ __forceinline__ uint4 row_piece(const float (&x)[C::EPT], int q) {
   if constexpr (C::BF16) {
+    uint32_t u[4];
 #pragma unroll
-    for (int q = 0; q < C::CPR; ++q) {
-      uint32_t u[4];
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const __nv_bfloat162 h2 = __floats2bfloat162_rn(p[4 * q + j].x, p[4 * q + j].y);
-        u[j] = *reinterpret_cast<const uint32_t *>(&h2);
-      }
-      *reinterpret_cast<uint4 *>(stage + (size_t)phys_chunk<C>(row, q) * 16) = make_uint4(u[0], u[1], u[2], u[3]);
+    for (int j = 0; j < 4; ++j) {
+      const __nv_bfloat162 h2 = __floats2bfloat162_rn(x[8 * q + 2 * j], x[8 * q + 2 * j + 1]);
+      u[j] = *reinterpret_cast<const uint32_t *>(&h2);
     }
+    return make_uint4(u[0], u[1], u[2], u[3]);
   } else {
-#pragma unroll
-    for (int q = 0; q < C::CPR; ++q)
-      *reinterpret_cast<float4 *>(stage + (size_t)phys_chunk<C>(row, q) * 16) =
-          make_float4(p[2 * q].x, p[2 * q].y, p[2 * q + 1].x, p[2 * q + 1].y);
+    return make_uint4(__float_as_uint(x[4 * q]), __float_as_uint(x[4 * q + 1]), __float_as_uint(x[4 * q + 2]),
+                      __float_as_uint(x[4 * q + 3]));
   }
 }
+
+constexpr int kBmCap = 1024;   // bit-map words of a CTA's tile range kept in shared memory (32768 tiles)
+constexpr int kChunkCap = kBmCap * 32 / 128;   // chunks of that range
+
+// Shared memory of decode_kernel: two input stages {payload slice, scale/zero words, pivot bytes}
+// filled by cp.async one chunk ahead, and one swizzled output stage from which the chunk leaves
+// with coalesced 16-byte stores.
+template <class C>
+struct DecSmem {
+  static constexpr int PAY = C::MAX_PAY + 32;
+  static constexpr int STAGE = PAY + C::TPC * 4 + C::TPC;
+  static constexpr int NST = 2;
+  static constexpr int ROWS = NST * STAGE;                  // offset of the swizzled output stage
+  static constexpr int TOTAL = ROWS + C::STAGE_BYTES;
+};
 
 template <class C>
 __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const Args a) {
-  extern __shared__ __align__(128) uint8_t smem[];   // one swizzled output stage
+  extern __shared__ __align__(128) uint8_t smem[];
+  using S = DecSmem<C>;
+  constexpr int WPC = C::TPC / 32;          // bit-map words per chunk
+  __shared__ uint32_t s_bm[kBmCap];         // bit map of this CTA's tiles (tail bits cleared)
+  __shared__ uint16_t s_chi[kChunkCap];     // higher-width tiles per chunk
   __shared__ uint8_t s_perm[kThreads];
   __shared__ uint2 s_cnt[kThreads / 32];
   __shared__ uint16_t s_rowoff[kThreads];
-  __shared__ uint8_t s_pv[kThreads];
   __shared__ uint32_t s_bad;
-  const uint32_t *sz32 = reinterpret_cast<const uint32_t *>(a.packed + a.off_sz);
-  const uint8_t *pivot = a.packed + a.off_pivot;
   const uint32_t *bitmap = reinterpret_cast<const uint32_t *>(a.packed + a.off_bitmap);
   const uint64_t n_chunks = (a.n_tiles + C::TPC - 1) / C::TPC;
   uint64_t c0, c1;
   cta_chunk_range(n_chunks, c0, c1);
+  const uint64_t t0 = c0 * C::TPC, t1 = c1 * C::TPC < a.n_tiles ? c1 * C::TPC : a.n_tiles;
+  const uint32_t nch = (uint32_t)(c1 - c0), nwords = nch * WPC;
+  if (nch > (uint32_t)kChunkCap) {   // more tiles per CTA than the format's tile limit allows with this grid
+    if (threadIdx.x == 0) atomicOr(a.status, 4u);
+    return;
+  }
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 
   // CTA 0 compares the received header with the one these parameters produce; its verdict travels
   // with the offset prefix, so a refused buffer leaves the output untouched.
@@ -826,136 +847,211 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const Args a) {
     refuse = s_bad != 0;
     if (refuse && threadIdx.x == 0) atomicOr(a.status, 1u /* TAHQ_DEV_BAD_HEADER */);
   }
-  // higher-width tiles before this CTA's range (Sec. 3.4 offsets), counted from the received bit map
+  // the bit map of this CTA's tiles goes to shared memory; count it per chunk and in total (Sec. 3.4)
   uint64_t hi_run = 0;
   {
     uint32_t n = 0;
-    if (a.mixed && !refuse) {
-      const uint64_t t0 = c0 * C::TPC, t1 = c1 * C::TPC < a.n_tiles ? c1 * C::TPC : a.n_tiles;
-      for (uint64_t wi = t0 / 32 + threadIdx.x; wi * 32 < t1; wi += kThreads) {
-        const uint64_t leftw = t1 - wi * 32;
-        n += __popc(__ldg(bitmap + wi) & (leftw >= 32 ? 0xffffffffu : ((1u << (uint32_t)leftw) - 1u)));
+    for (uint32_t wi = threadIdx.x; wi < nwords; wi += kThreads) {
+      uint32_t word = 0;
+      const uint64_t first = t0 + 32ull * wi;
+      if (a.mixed && !refuse && first < t1) {
+        const uint64_t leftw = t1 - first;
+        word = __ldg(bitmap + t0 / 32 + wi) & (leftw >= 32 ? 0xffffffffu : ((1u << (uint32_t)leftw) - 1u));
       }
+      s_bm[wi] = word;
+      n += __popc(word);
     }
-    const uint32_t mine = block_sum(n);
+    const uint32_t mine = block_sum(n);   // barrier inside: s_bm is complete
+    for (uint32_t ci = threadIdx.x; ci < nch; ci += kThreads) {
+      uint32_t m = 0;
+#pragma unroll
+      for (int w = 0; w < WPC; ++w) m += __popc(s_bm[ci * WPC + w]);
+      s_chi[ci] = (uint16_t)m;
+    }
     bool stop;
-    hi_run = cta_exclusive_prefix(a, mine, refuse, stop);
+#if defined(TAHQ_ABLATE) && (TAHQ_ABLATE & 4)
+    stop = false; hi_run = 0; __syncthreads();
+#else
+    hi_run = cta_exclusive_prefix(a, mine, refuse, stop);   // barriers inside: s_chi is complete
+#endif
     if (blockIdx.x == gridDim.x - 1 && threadIdx.x == 0 && a.mixed && !stop &&
         hi_run + mine != a.n_groups * a.k_hi)
       atomicOr(a.status, 2u /* TAHQ_DEV_BAD_BITMAP */);
     if (stop) return;
   }
 
-  for (uint64_t c = c0; c < c1; ++c) {
-    const uint64_t tile0 = c * C::TPC;
+  // One thread moves a chunk's payload slice (from the 16-byte boundary below it), scale/zero words
+  // and pivot bytes with three bulk copies that complete on the stage's mbarrier.
+  __shared__ __align__(8) unsigned long long s_bar[S::NST];
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < S::NST; ++i) mbar_init(&s_bar[i], 1);
+    mbar_init_fence();
+  }
+  __syncthreads();
+  auto issue = [&](uint32_t ci, uint64_t hi_before, int stg) {
+    uint8_t *st = smem + (size_t)stg * S::STAGE;
+    const uint64_t tile0 = t0 + (uint64_t)ci * C::TPC;
+    const uint64_t left = a.n_tiles - tile0;
+    const uint32_t nv = left < (uint64_t)C::TPC ? (uint32_t)left : (uint32_t)C::TPC;
+    const uint64_t goff = (uint64_t)(C::G / 8) * ((uint64_t)a.lo * tile0 + hi_before);
+    uint64_t bytes = (uint64_t)(C::G / 8) * ((uint64_t)a.lo * nv + s_chi[ci]);
+    if (goff + bytes > a.payload_bytes) bytes = goff < a.payload_bytes ? a.payload_bytes - goff : 0;   // corrupt bit map
+    const uint32_t npay = (uint32_t)(((goff & 15ull) + bytes + 15) & ~15ull);
+    const uint32_t nsz = (nv * 4 + 15) & ~15u, npv = (nv + 15) & ~15u;
+    fence_async_proxy();   // earlier reads of this stage are ordered before the asynchronous writes
+    mbar_expect_tx(&s_bar[stg], npay + nsz + npv);
+    if (npay) bulk_copy_g2s(st, a.packed + a.off_payload + (goff & ~15ull), npay, &s_bar[stg]);
+    bulk_copy_g2s(st + S::PAY, a.packed + a.off_sz + 4 * tile0, nsz, &s_bar[stg]);
+    bulk_copy_g2s(st + S::PAY + C::TPC * 4, a.packed + a.off_pivot + tile0, npv, &s_bar[stg]);
+  };
+
+  uint8_t *ostage = smem + S::ROWS;
+  // this thread's pieces of the coalesced copy-out: chunk index i*kThreads + tid sits in row i*(kThreads/CPR) + tid/CPR
+  const uint8_t *co_src = ostage + (size_t)((int)threadIdx.x ^ swz<C>((int)threadIdx.x / C::CPR)) * 16;
+#if defined(TAHQ_ABLATE) && (TAHQ_ABLATE & 8)
+  long long tk[6] = {0, 0, 0, 0, 0, 0}; long long tprev = clock64();
+#define TAHQ_TICK(i) do { long long now_ = clock64(); tk[i] += now_ - tprev; tprev = now_; } while (0)
+#else
+#define TAHQ_TICK(i) do {} while (0)
+#endif
+  if (nch && threadIdx.x == 0) issue(0, hi_run, 0);
+  int stage = 0;
+  unsigned phases = 0;   // bit s = parity of stage s's mbarrier phase to wait for
+  for (uint32_t ci = 0; ci < nch; ++ci) {
+    const uint32_t hi_here = s_chi[ci];
+    if (ci + 1 < nch && threadIdx.x == 0)   // the next chunk goes into the other stage (everyone left it last iteration)
+      issue(ci + 1, hi_run + hi_here, stage ^ 1);
+    TAHQ_TICK(0);
+    if (!mbar_wait(&s_bar[stage], (phases >> stage) & 1u)) atomicOr(a.status, 4u /* TAHQ_DEV_TIMEOUT */);   // chunk ci has landed
+    phases ^= 1u << stage;
+    TAHQ_TICK(1);
+
+    const uint8_t *st = smem + (size_t)stage * S::STAGE;
+    const uint64_t tile0 = t0 + (uint64_t)ci * C::TPC;
     const uint64_t left = a.n_tiles - tile0;
     const uint32_t nvalid = left < (uint64_t)C::TPC ? (uint32_t)left : (uint32_t)C::TPC;
-    const uint32_t own = threadIdx.x / C::LPT;
     const uint64_t goff = (uint64_t)(C::G / 8) * ((uint64_t)a.lo * tile0 + hi_run);
-    const uint8_t *pay = a.packed + a.off_payload + goff;
-    float2 x[C::EPT / 2];
-    bool hi1 = false;
-    if (a.mixed && own < nvalid) hi1 = (__ldg(bitmap + (tile0 + own) / 32) >> ((tile0 + own) & 31)) & 1u;
-    uint32_t chunk_bytes;
+    const uint8_t *pay = st + (goff & 15ull);
+    const uint32_t *sz = reinterpret_cast<const uint32_t *>(st + S::PAY);
+    const uint8_t *pv = st + S::PAY + C::TPC * 4;
+    const bool fits = goff + (uint64_t)(C::G / 8) * ((uint64_t)a.lo * nvalid + hi_here) <= a.payload_bytes;
+    hi_run += hi_here;
 
     if constexpr (C::LPT == 1) {
-      // phase 1: thread r reads tile r's pivot byte; the CTA regroups tiles by (transformed?, width)
-      const uint32_t pv1 = own < nvalid ? __ldg(pivot + tile0 + own) : 0u;
-      const Regroup rg = regroup(((pv1 & 0x80u) ? 2 : 0) | (hi1 ? 1 : 0), s_perm, s_cnt, [&](const Regroup &r) {
+      // phase 1: thread r reads tile r's pivot byte and width bit; the CTA regroups tiles by (transformed?, width)
+      const uint32_t pv1 = threadIdx.x < nvalid ? pv[threadIdx.x] : 0u;
+      const uint32_t hi1 = (s_bm[ci * WPC + warp] >> lane) & 1u;
+      const Regroup rg = regroup(((pv1 & 0x80u) ? 2 : 0) | (int)hi1, s_perm, s_cnt, [&](const Regroup &r) {
         s_rowoff[threadIdx.x] = (uint16_t)((C::G / 8) * (a.lo * threadIdx.x + r.hi_before));
-        s_pv[threadIdx.x] = (uint8_t)pv1;
       });
-      chunk_bytes = (C::G / 8) * (a.lo * nvalid + rg.total_hi);
-      hi_run += rg.total_hi;
-      const bool fits = goff + chunk_bytes <= a.payload_bytes;   // false only for a corrupt bit map
-      // phase 2
+      // phase 2: this thread now owns tile `src` of the chunk
+      TAHQ_TICK(2);
       const int src = rg.src;
       const bool flag = rg.cls & 2;
-      const uint32_t b = a.lo + (rg.cls & 1);
-      const uint64_t tile = tile0 + src;
       if ((uint32_t)src < nvalid && fits) {
-        const uint32_t szw = __ldg(sz32 + tile);
+        const uint32_t szw = sz[src];
         const float s = __half2float(__ushort_as_half((unsigned short)(szw & 0xffffu)));
         const float z = __half2float(__ushort_as_half((unsigned short)(szw >> 16)));
-        load_dequant<C::EPT>(reinterpret_cast<const uint32_t *>(pay + s_rowoff[src]), b, s, z, x);
-      } else {
+        float x[C::EPT];
+#if defined(TAHQ_ABLATE) && (TAHQ_ABLATE & 1)
 #pragma unroll
-        for (int i = 0; i < C::EPT / 2; ++i) x[i] = f2(0.0f);
-      }
-      if (flag) {   // (1/sqrt G) H_G^T = the same butterfly
-        butterfly2<C::EPT / 2>(x);
+        for (int k = 0; k < C::EPT; ++k) x[k] = s + z * k;
+#else
+        load_dequant<C::EPT>(pay + s_rowoff[src], a.lo + (rg.cls & 1), s, z, x);
+#endif
+        if (flag) {   // (1/sqrt G) H_G^T = the same butterfly
+          butterfly<C::EPT>(x);
 #pragma unroll
-        for (int i = 0; i < C::EPT / 2; ++i) x[i] = mul2(x[i], f2(hadamard_scale<C>()));
-      }
-      stage_row<C>(smem, src, x);
-      if (flag) {   // un-swap coordinates 0 and d in the staged row
-        asm volatile("" ::: "memory");
-        row_swap_0_d<C, !C::BF16>(smem, src, s_pv[src] & 0x7f);
+          for (int k = 0; k < C::EPT; ++k) x[k] = x[k] * hadamard_scale<C>();
+        }
+        uint8_t *orow = ostage + (size_t)src * C::ROWB;
+        const int sx = swz<C>(src) * 16;
+#pragma unroll
+        for (int q = 0; q < C::CPR; ++q) *reinterpret_cast<uint4 *>(orow + ((q * 16) ^ sx)) = row_piece<C>(x, q);
+        if (flag) {   // un-swap coordinates 0 and d in the staged row
+          asm volatile("" ::: "memory");
+          row_swap_0_d<C, !C::BF16>(ostage, src, pv[src] & 0x7f);
+        }
       }
     } else {
       const int half = threadIdx.x & 1;
-      const uint64_t tile = tile0 + own;
+      const uint32_t own = threadIdx.x >> 1;
+      const bool hi1 = (s_bm[ci * WPC + (own >> 5)] >> (own & 31)) & 1u;
       uint32_t hi_before, total_hi, tiles16;
       pair_scan(hi1, reinterpret_cast<uint32_t *>(s_cnt), hi_before, total_hi, tiles16);
-      chunk_bytes = (C::G / 8) * (a.lo * nvalid + total_hi);
-      hi_run += total_hi;
-      const bool fits = goff + chunk_bytes <= a.payload_bytes;
       const uint32_t b = a.lo + (hi1 ? 1u : 0u);
       const uint32_t row_off = (C::G / 8) * (a.lo * own + hi_before) + half * (C::EPT / 8) * b;
-      uint32_t pv = 0;
-      if (own < nvalid && fits) {
-        const uint32_t szw = __ldg(sz32 + tile);
+      const bool live = own < nvalid && fits;
+      float x[C::EPT];
+      uint32_t pvb = 0;
+      if (live) {
+        const uint32_t szw = sz[own];
         const float s = __half2float(__ushort_as_half((unsigned short)(szw & 0xffffu)));
         const float z = __half2float(__ushort_as_half((unsigned short)(szw >> 16)));
-        pv = __ldg(pivot + tile);
-        load_dequant<C::EPT>(reinterpret_cast<const uint32_t *>(pay + row_off), b, s, z, x);
+        pvb = pv[own];
+        load_dequant<C::EPT>(pay + row_off, b, s, z, x);
       } else {
 #pragma unroll
-        for (int i = 0; i < C::EPT / 2; ++i) x[i] = f2(0.0f);
+        for (int k = 0; k < C::EPT; ++k) x[k] = 0.0f;
       }
-      const bool flag = (pv & 0x80u) != 0;
+      const bool flag = (pvb & 0x80u) != 0;
       const unsigned fm = __ballot_sync(kFull, flag);
       if (flag) {
-        const int d = pv & 0x7f;
-        butterfly2<C::EPT / 2>(x);
+        const int d = pvb & 0x7f;
+        butterfly<C::EPT>(x);
 #pragma unroll
-        for (int i = 0; i < C::EPT / 2; ++i) {   // last stage: across the two lanes of the tile
-          const float px = __shfl_xor_sync(fm, x[i].x, 1), py = __shfl_xor_sync(fm, x[i].y, 1);
-          x[i] = half ? make_float2(px - x[i].x, py - x[i].y) : make_float2(x[i].x + px, x[i].y + py);
+        for (int k = 0; k < C::EPT; ++k) {   // last stage: across the two lanes of the tile
+          const float p = __shfl_xor_sync(fm, x[k], 1);
+          x[k] = half ? (p - x[k]) : (x[k] + p);
         }
 #pragma unroll
-        for (int i = 0; i < C::EPT / 2; ++i) x[i] = mul2(x[i], f2(hadamard_scale<C>()));
-        const int lane = threadIdx.x & 31, owner = d / C::EPT, dl = d % C::EPT;
-        float mine = x[0].x;   // un-swap coordinates 0 and d (d may sit in the other lane)
+        for (int k = 0; k < C::EPT; ++k) x[k] = x[k] * hadamard_scale<C>();
+        const int owner = d / C::EPT, dl = d % C::EPT;
+        float mine = x[0];   // un-swap coordinates 0 and d (d may sit in the other lane)
 #pragma unroll
-        for (int k = 1; k < C::EPT; ++k) mine = (k == dl) ? ((k & 1) ? x[k >> 1].y : x[k >> 1].x) : mine;
-        const float x0 = __shfl_sync(fm, x[0].x, lane & ~1);
+        for (int k = 1; k < C::EPT; ++k) mine = (k == dl) ? x[k] : mine;
+        const float x0 = __shfl_sync(fm, x[0], lane & ~1);
         const float xd = __shfl_sync(fm, mine, (lane & ~1) + owner);
         if (half == owner) {
 #pragma unroll
-          for (int k = 0; k < C::EPT; ++k) {
-            if (k & 1) x[k >> 1].y = (k == dl) ? x0 : x[k >> 1].y;
-            else x[k >> 1].x = (k == dl) ? x0 : x[k >> 1].x;
-          }
+          for (int k = 0; k < C::EPT; ++k) x[k] = (k == dl) ? x0 : x[k];
         }
-        if (half == 0) x[0].x = xd;
+        if (half == 0) x[0] = xd;
       }
-      stage_row<C>(smem, (int)threadIdx.x, x);
-    }
-
-    // the chunk leaves with coalesced 16-byte stores
-    __syncthreads();
-    const uint32_t valid_bytes = nvalid * C::G * C::ESZ;
-    uint8_t *gout = a.out + tile0 * (uint64_t)(C::G * C::ESZ);
 #pragma unroll
-    for (int i = 0; i < C::CPR; ++i) {
-      const int ci = i * kThreads + (int)threadIdx.x;
-      if ((uint32_t)ci * 16u < valid_bytes)
-        *reinterpret_cast<uint4 *>(gout + (size_t)ci * 16) =
-            *reinterpret_cast<const uint4 *>(smem + (size_t)(ci ^ swz<C>(ci / C::CPR)) * 16);
+      for (int q = 0; q < C::CPR; ++q)
+        *reinterpret_cast<uint4 *>(ostage + (size_t)phys_chunk<C>((int)threadIdx.x, q) * 16) = row_piece<C>(x, q);
     }
-    __syncthreads();
+    TAHQ_TICK(3);
+    stage ^= 1;
+    __syncthreads();   // the chunk is staged; everyone is done with this input stage
+    TAHQ_TICK(4);
+#if defined(TAHQ_ABLATE) && (TAHQ_ABLATE & 2)
+    if (fits && a.lo == 99) {
+#else
+    if (fits) {   // the chunk leaves with coalesced 16-byte stores
+#endif
+      uint8_t *gout = a.out + tile0 * (uint64_t)(C::G * C::ESZ) + (size_t)threadIdx.x * 16;
+      if (nvalid == (uint32_t)C::TPC) {
+#pragma unroll
+        for (int i = 0; i < C::CPR; ++i)
+          *reinterpret_cast<uint4 *>(gout + (size_t)i * kThreads * 16) =
+              *reinterpret_cast<const uint4 *>(co_src + (size_t)i * kThreads * 16);
+      } else {
+        const uint32_t valid_bytes = nvalid * C::G * C::ESZ;
+#pragma unroll
+        for (int i = 0; i < C::CPR; ++i)
+          if ((uint32_t)(i * kThreads + (int)threadIdx.x) * 16u < valid_bytes)
+            *reinterpret_cast<uint4 *>(gout + (size_t)i * kThreads * 16) =
+                *reinterpret_cast<const uint4 *>(co_src + (size_t)i * kThreads * 16);
+      }
+    }
+    TAHQ_TICK(5);
   }
+#if defined(TAHQ_ABLATE) && (TAHQ_ABLATE & 8)
+  if (threadIdx.x == 0) for (int i = 0; i < 6; ++i) a.cand[blockIdx.x * 8 + i] = (unsigned long long)tk[i];
+  if (threadIdx.x == 0) a.cand[blockIdx.x * 8 + 6] = nch;
+#endif
 }
 
 }  // namespace tahq
