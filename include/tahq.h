@@ -40,7 +40,8 @@ typedef enum {
   TAHQ_ERR_UNSUPPORTED = 2,      /* valid in the format but not built (e.g. tile < 32)          */
   TAHQ_ERR_BUFFER_TOO_SMALL = 3, /* packed_cap / packed_bytes / ws_cap below the bound          */
   TAHQ_ERR_MISALIGNED = 4,       /* a device pointer is not 16-byte aligned                     */
-  TAHQ_ERR_CUDA = 5              /* a CUDA runtime call (launch, memset) failed                 */
+  TAHQ_ERR_CUDA = 5,             /* a CUDA runtime call (launch, memset) failed                 */
+  TAHQ_ERR_TOO_LARGE = 6         /* tahq_encode_noalloc: needs more scratch than is built in    */
 } tahq_status;
 
 typedef enum { TAHQ_F32 = 0, TAHQ_BF16 = 1 } tahq_dtype;
@@ -132,6 +133,36 @@ tahq_status tahq_encode(const tahq_params *p, const void *d_in, void *d_packed, 
  */
 tahq_status tahq_decode(const tahq_params *p, const void *d_packed, size_t packed_bytes, void *d_out,
                         void *d_ws, size_t ws_cap, tahq_stream stream);
+
+/*
+ * Encode without a caller-provided workspace (the paper has no counterpart; this is a convenience of
+ * the library).  Same operation, same bytes in d_packed as tahq_encode, but the scratch memory lives
+ * in a fixed TAHQ_NOALLOC_SCRATCH_BYTES (8 MiB) buffer that is part of the library image on every GPU
+ * that loads it, so the call neither needs a workspace pointer nor allocates or frees anything.
+ *
+ * Who needs this: code that is handed device pointers but owns no allocator and may not call
+ * cudaMalloc -- a communication plug-in working on buffers registered by its host framework, a
+ * process whose device memory was carved up in advance by a pool it cannot ask, or a step that runs
+ * where an allocation would force a device-wide synchronisation.
+ *
+ * Limits and rules
+ *   - Accepts exactly the configurations with tahq_workspace_bound(p) <= TAHQ_NOALLOC_SCRATCH_BYTES
+ *     (e.g. 8192 x 4096 elements at tile 64 needs 3.2 MB); anything larger returns
+ *     TAHQ_ERR_TOO_LARGE and enqueues nothing.
+ *   - The first call on each device looks up the device address of the built-in buffer (a host-side
+ *     set-up step, done once per device with that device current).  Make that first call before any
+ *     stream capture begins.
+ *   - All calls on one device share the one buffer.  It keeps the previous call's contents; each call
+ *     clears the part that must start at zero on the given stream.  Two calls that may overlap on the
+ *     GPU (different streams without an ordering between them) race on it: order them, or use
+ *     tahq_encode with separate workspaces.
+ *   - The device status word of the call cannot be read back by the caller; use tahq_encode when that
+ *     is needed.
+ * Errors: as tahq_encode, plus TAHQ_ERR_TOO_LARGE.
+ */
+#define TAHQ_NOALLOC_SCRATCH_BYTES (8u << 20)
+tahq_status tahq_encode_noalloc(const tahq_params *p, const void *d_in, void *d_packed, size_t packed_cap,
+                                tahq_stream stream);
 
 /* Static string for a status code. */
 const char *tahq_status_string(tahq_status s);

@@ -67,6 +67,7 @@ class TahqError(RuntimeError):
 
 
 EXPORTS = ["tahq_packed_bound", "tahq_packed_layout", "tahq_workspace_bound", "tahq_encode", "tahq_decode",
+           "tahq_encode_noalloc",
            "tahq_status_string", "tahq_last_launch_count", "tahq_profile", "tahq_profile_read"]
 
 _lib = None
@@ -88,6 +89,8 @@ def lib() -> C.CDLL:
         L.tahq_workspace_bound.restype = C.c_size_t
         L.tahq_encode.argtypes = [pp, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p, C.c_size_t, C.c_void_p]
         L.tahq_encode.restype = C.c_int
+        L.tahq_encode_noalloc.argtypes = [pp, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+        L.tahq_encode_noalloc.restype = C.c_int
         L.tahq_decode.argtypes = [pp, C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
         L.tahq_decode.restype = C.c_int
         L.tahq_status_string.argtypes = [C.c_int]
@@ -150,6 +153,22 @@ def tahq_encode(p: Params, d_in: int, d_packed: int, packed_cap: int, d_ws: int,
     """Raw call: device addresses as integers, returns the tahq_status."""
     pc = p.c()
     return int(lib().tahq_encode(C.byref(pc), d_in, d_packed, packed_cap, d_ws, ws_cap, stream))
+
+
+NOALLOC_SCRATCH_BYTES = 8 << 20
+ERR_TOO_LARGE = 6
+
+
+def tahq_encode_noalloc(p: Params, d_in: int, d_packed: int, packed_cap: int, stream: int) -> int:
+    """Raw call of the workspace-free encode: scratch comes from the library's built-in 8 MiB buffer.
+
+    For callers that hold device pointers but cannot allocate (no allocator of their own, memory
+    carved up in advance, or a place where an allocation would synchronise the device).  Returns the
+    tahq_status; ERR_TOO_LARGE when workspace_bound(p) exceeds NOALLOC_SCRATCH_BYTES.  Calls on one
+    device share the buffer, so calls that could overlap on the GPU must be ordered by the caller.
+    """
+    pc = p.c()
+    return int(lib().tahq_encode_noalloc(C.byref(pc), d_in, d_packed, packed_cap, stream))
 
 
 def tahq_decode(p: Params, d_packed: int, packed_bytes: int, d_out: int, d_ws: int, ws_cap: int, stream: int) -> int:

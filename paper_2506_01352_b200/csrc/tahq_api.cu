@@ -239,6 +239,12 @@ static tahq_status decode_t(const Plan &pl, const Args &a, cudaStream_t st) {
 
 static bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// Scratch for tahq_encode_noalloc: part of the library image, resident on every GPU that loads it.
+// In host code this name is only a handle; the device address is looked up once per device.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[TAHQ_NOALLOC_SCRATCH_BYTES];
+static void *g_noalloc_addr[64];
+static std::atomic<int> g_noalloc_ready[64];
+
 }  // namespace tahq
 
 using namespace tahq;
@@ -310,6 +316,26 @@ tahq_status tahq_decode(const tahq_params *p, const void *d_packed, size_t packe
   }
 }
 
+tahq_status tahq_encode_noalloc(const tahq_params *p, const void *d_in, void *d_packed, size_t packed_cap,
+                                tahq_stream stream) {
+  g_launches = 0;
+  Plan pl;
+  const tahq_status s = make_plan(p, &pl);
+  if (s != TAHQ_OK) return s;
+  if (pl.ws_total > (uint64_t)TAHQ_NOALLOC_SCRATCH_BYTES) return TAHQ_ERR_TOO_LARGE;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return TAHQ_ERR_CUDA;
+  if (!g_noalloc_ready[dev].load(std::memory_order_acquire)) {
+    // set-up, once per device, with that device current: the device address behind the symbol
+    void *ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_noalloc_scratch) != cudaSuccess || !ptr) return TAHQ_ERR_CUDA;
+    g_noalloc_addr[dev] = ptr;
+    g_noalloc_ready[dev].store(1, std::memory_order_release);
+  }
+  // tahq_encode clears the head of the workspace (status, flags, histograms, counters) on the stream
+  return tahq_encode(p, d_in, d_packed, packed_cap, g_noalloc_addr[dev], TAHQ_NOALLOC_SCRATCH_BYTES, stream);
+}
+
 const char *tahq_status_string(tahq_status s) {
   switch (s) {
     case TAHQ_OK: return "ok";
@@ -318,6 +344,7 @@ const char *tahq_status_string(tahq_status s) {
     case TAHQ_ERR_BUFFER_TOO_SMALL: return "buffer too small";
     case TAHQ_ERR_MISALIGNED: return "pointer not 16-byte aligned";
     case TAHQ_ERR_CUDA: return "CUDA runtime error";
+    case TAHQ_ERR_TOO_LARGE: return "tensor needs more scratch than the built-in buffer of tahq_encode_noalloc";
   }
   return "unknown status";
 }
