@@ -29,7 +29,12 @@ L2_BYTES = 126e6
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch, from the ncu captures summarised under
 # profiles/ (same kernel, same workload); None until a capture exists for that kernel.
-NCU_TRAFFIC_BYTES = {}
+NCU_TRAFFIC_BYTES = {
+    # profiles/ncu_full_c3_llama7b_b3800_tile_kernels.md (cold-cache capture, one launch)
+    ("stats", "c3_llama7b", 3800, 64): 68.03e6,
+    ("quant_pack", "c3_llama7b", 3800, 64): 72.53e6,
+    ("decode", "c3_llama7b", 3800, 64): 27.94e6,
+}
 
 
 def parse_args():
