@@ -51,7 +51,8 @@ enum {
   TAHQ_DEV_OK = 0,
   TAHQ_DEV_BAD_HEADER = 1,       /* decode: the buffer's header does not match the parameters   */
   TAHQ_DEV_BAD_BITMAP = 2,       /* decode: bit map population does not match the payload size  */
-  TAHQ_DEV_TIMEOUT = 4           /* a bounded device-side wait ran out                          */
+  TAHQ_DEV_TIMEOUT = 4,          /* a bounded device-side wait ran out                          */
+  TAHQ_DEV_INTERNAL = 8          /* encode: a screening bound of the tile selection was violated */
 };
 
 /*
@@ -74,7 +75,7 @@ typedef struct {
   float tau;                 /* outlier threshold of Eq. 3 (paper: 2.0; 0 = always transform,
                                 +inf = never)                                                    */
   float eps_l1;              /* epsilon  of Eq. 1 (1e-8f)                                        */
-  float eps_log;             /* varsigma of Eq. 2 (1e-8f)                                        */
+  float eps_log;             /* varsigma of Eq. 2 (1e-8f); a positive normal binary32 number     */
   float eps_ratio;           /* varrho   of Eq. 3 (1e-8f)                                        */
   uint32_t rounding;         /* 0 = round-half-even; 1 = stochastic (Philox4x32-10 keyed by seed,
                                 counter = element index / 4)                                     */

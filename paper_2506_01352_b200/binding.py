@@ -16,7 +16,7 @@ from . import build as _build
 
 F32, BF16 = 0, 1
 OK = 0
-DEV_OK, DEV_BAD_HEADER, DEV_BAD_BITMAP, DEV_TIMEOUT = 0, 1, 2, 4
+DEV_OK, DEV_BAD_HEADER, DEV_BAD_BITMAP, DEV_TIMEOUT, DEV_INTERNAL = 0, 1, 2, 4, 8
 
 
 class _Params(C.Structure):

@@ -43,7 +43,7 @@ struct Plan {
   bool direct;            // small ranking groups: select straight from the scores
   uint32_t cpg, cand_cap;
   // workspace offsets
-  uint64_t ws_flags, ws_ncand, ws_done, ws_hist, ws_zero_end, ws_scores, ws_theta, ws_cand, ws_total;
+  uint64_t ws_flags, ws_ncand, ws_done, ws_nabove, ws_hist, ws_zero_end, ws_scores, ws_theta, ws_cand, ws_total;
 };
 
 static uint64_t up(uint64_t x, uint64_t a) { return (x + a - 1) / a * a; }
@@ -58,7 +58,8 @@ static tahq_status make_plan(const tahq_params *p, Plan *pl) {
   if (p->tokens % S) return TAHQ_ERR_INVALID_ARG;
   const uint32_t beta = p->budget_millibits;
   if (beta < 2000 || beta > 8000) return TAHQ_ERR_INVALID_ARG;
-  if (!(p->tau >= 0.0f) || !(p->eps_l1 >= 0.0f) || !(p->eps_log >= 0.0f) || !(p->eps_ratio >= 0.0f))
+  // varsigma must be a positive normal number: p + varsigma is split into exponent and mantissa
+  if (!(p->tau >= 0.0f) || !(p->eps_l1 >= 0.0f) || !(p->eps_log >= 1.17549435e-38f) || !(p->eps_ratio >= 0.0f))
     return TAHQ_ERR_INVALID_ARG;
   const uint64_t M = p->hidden / G;
   if (p->tokens > (1ull << 40) / M) return TAHQ_ERR_INVALID_ARG;
@@ -94,6 +95,7 @@ static tahq_status make_plan(const tahq_params *p, Plan *pl) {
   pl->ws_flags = o;  o += 8ull * kMaxGrid;
   pl->ws_ncand = o;  o = up(o + (hist ? 4 * L.n_groups : 0), 256);
   pl->ws_done = o;   o = up(o + (hist ? 4 * L.n_groups : 0), 256);
+  pl->ws_nabove = o; o = up(o + (hist ? 4 * L.n_groups : 0), 256);
   pl->ws_hist = o;   o += hist ? 4ull * kBins * L.n_groups : 0;
   pl->ws_zero_end = o;                                      // [0, ws_zero_end) is cleared by every encode
   pl->ws_scores = o; o = up(o + (pl->mixed ? 4 * L.n_tiles : 0), 256);
@@ -149,6 +151,9 @@ static void fill_args(const tahq_params *p, const Plan &pl, uint8_t *ws, Args *a
   a->hist = reinterpret_cast<uint32_t *>(ws + pl.ws_hist);
   a->scores = reinterpret_cast<float *>(ws + pl.ws_scores);
   a->done = reinterpret_cast<uint32_t *>(ws + pl.ws_done);
+  a->nabove = reinterpret_cast<uint32_t *>(ws + pl.ws_nabove);
+  a->bf16 = p->dtype == TAHQ_BF16;
+  a->tile = p->tile;
   a->flags = reinterpret_cast<unsigned long long *>(ws + pl.ws_flags);
   a->theta = reinterpret_cast<unsigned long long *>(ws + pl.ws_theta);
   a->cand = reinterpret_cast<unsigned long long *>(ws + pl.ws_cand);
@@ -180,7 +185,7 @@ static int prepare(K kernel, int smem, const DevInfo &d, std::atomic<int> *cache
 }
 
 template <class C> struct Stages {
-  static constexpr int STATS = (C::ROWB == 64) ? 3 : 2;
+  static constexpr int STATS = (C::ROWB == 256) ? 2 : TAHQ_STATS_NST;
   static constexpr int QUANT = (C::ROWB == 256) ? 2 : (C::ROWB == 128 ? 2 : 3);
 };
 

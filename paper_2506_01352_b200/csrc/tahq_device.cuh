@@ -271,41 +271,146 @@ __device__ __forceinline__ void load_abs_oct_pair(const uint8_t *stage, int row,
   }
 }
 
+// log2 of a positive normal number, exponent + u*Q(u) as in lg2_poly, with the exponent and the
+// mantissa split done by multiply-adds so that everything runs on the FMA pipe (the ALU pipe has
+// half its rate and is the busier one):  (x * 512) >> 32 is the biased exponent eb, placed into the
+// mantissa of 2^23 by the addend of the same integer multiply-add; 2^-E is built as a bit pattern
+// by one more integer multiply-add, and u = x * 2^-E - 1 is exact (so is every step: the result has
+// the same bits as lg2_poly).
+__device__ __forceinline__ float lg2_fma(float x) {
+  const uint32_t xi = __float_as_uint(x);
+  uint32_t ebm;
+  asm("mad.hi.u32 %0, %1, 512, 0x4B000000;" : "=r"(ebm) : "r"(xi));   // bits of 2^23 + eb
+  const float e = __uint_as_float(ebm) - 8388735.0f;                   // eb - 127
+  const uint32_t sb = ebm * 0xFF800000u + 0x7F000000u;                 // (254 - eb) << 23: bits of 2^-E
+  const float u = __fmaf_rn(x, __uint_as_float(sb), -1.0f);
+  float q = -0x1.a762d6p-6f;
+  q = __fmaf_rn(q, u, 0x1.f2e252p-4f);
+  q = __fmaf_rn(q, u, -0x1.1c9334p-2f);
+  q = __fmaf_rn(q, u, 0x1.d487c6p-2f);
+  q = __fmaf_rn(q, u, -0x1.6fb0bcp-1f);
+  q = __fmaf_rn(q, u, 0x1.714aa0p+0f);
+  return __fmaf_rn(u, q, e);
+}
+
+// Magnitudes of eight consecutive elements of a row.
+template <class C>
+__device__ __forceinline__ void load_abs_oct(const uint8_t *stage, int row, int o, float (&v)[8]) {
+  if constexpr (C::BF16) {
+    const uint4 w = *reinterpret_cast<const uint4 *>(stage + (size_t)phys_chunk<C>(row, o) * 16);
+    const uint32_t u[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j)   // clear both sign bits at once, widen on the FMA pipe
+      bf2_add_f32(u[j] & 0x7fff7fffu, -0.0f, v[2 * j], v[2 * j + 1]);
+  } else {
+    load_oct<C>(stage, row, o, v);
+#pragma unroll
+    for (int k = 0; k < 8; ++k) v[k] = fabsf(v[k]);
+  }
+}
+
 // Entropy score of the tile this thread (pair) owns: -sum p log2(p + varsigma), p = |a| / (L1 + eps).
+// Two streaming passes over the row in shared memory, eight elements at a time.
 template <class C>
 __device__ __forceinline__ float tile_score(const uint8_t *stage, float eps_l1, float eps_log) {
-  constexpr int NP = C::NOCT / 2;
   const int row = (int)threadIdx.x;
-  float2 a[NP][8];
   float part[C::NOCT];
 #pragma unroll
-  for (int p = 0; p < NP; ++p) {
-    load_abs_oct_pair<C>(stage, row, p, a[p]);
-    const float2 s = tree8x2(a[p]);
-    part[2 * p] = s.x;
-    part[2 * p + 1] = s.y;
+  for (int o = 0; o < C::NOCT; ++o) {
+    float v[8];
+    load_abs_oct<C>(stage, row, o, v);
+    part[o] = tree8(v);
   }
   float L1 = tree<C::NOCT>(part);
   if constexpr (C::LPT == 2) L1 = L1 + __shfl_xor_sync(kFull, L1, 1);
   const float inv = __fdiv_rn(1.0f, L1 + eps_l1);
-  const float2 eps = f2(eps_log);
 #pragma unroll
-  for (int p = 0; p < NP; ++p) {
-    float2 t[8];
+  for (int o = 0; o < C::NOCT; ++o) {
+    float v[8];
+    load_abs_oct<C>(stage, row, o, v);
 #pragma unroll
     for (int k = 0; k < 8; ++k) {
-      const float2 pk = f2(a[p][k].x * inv, a[p][k].y * inv);   // scalar: pk is added to below
-      t[k] = mul2(pk, lg2_poly2(add2(pk, eps)));
+      const float p = v[k] * inv;
+      v[k] = p * lg2_fma(p + eps_log);
     }
-    // first tree level with scalar adds (its operands are packed products), the rest packed
-    const float2 s01 = f2(t[0].x + t[1].x, t[0].y + t[1].y), s23 = f2(t[2].x + t[3].x, t[2].y + t[3].y);
-    const float2 s45 = f2(t[4].x + t[5].x, t[4].y + t[5].y), s67 = f2(t[6].x + t[7].x, t[6].y + t[7].y);
-    const float2 s = add2(add2(s01, s23), add2(s45, s67));
-    part[2 * p] = s.x;
-    part[2 * p + 1] = s.y;
+    part[o] = tree8(v);
   }
   float S = tree<C::NOCT>(part);
   if constexpr (C::LPT == 2) S = S + __shfl_xor_sync(kFull, S, 1);
+  return 0.0f - S;
+}
+
+// ---- Screening score: the same sums with the hardware's approximate log2 (one MUFU instruction
+// instead of ten FMA-pipe instructions per element).  It is only used to decide which tiles are
+// far enough from a group's threshold to be classified without their exact score; see select_kernel.
+__device__ __forceinline__ float lg2_approx(float x) {
+  float y;
+  asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+template <class C>
+__device__ __forceinline__ float tile_score_screen(const uint8_t *stage, float eps_l1, float eps_log) {
+  const int row = (int)threadIdx.x;
+  float part[C::NOCT];
+#pragma unroll
+  for (int o = 0; o < C::NOCT; ++o) {
+    float v[8];
+    load_abs_oct<C>(stage, row, o, v);
+    part[o] = tree8(v);
+  }
+  float L1 = tree<C::NOCT>(part);
+  if constexpr (C::LPT == 2) L1 = L1 + __shfl_xor_sync(kFull, L1, 1);
+  const float inv = __fdiv_rn(1.0f, L1 + eps_l1);
+#pragma unroll
+  for (int o = 0; o < C::NOCT; ++o) {
+    float v[8];
+    load_abs_oct<C>(stage, row, o, v);
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+      const float p = v[k] * inv;
+      v[k] = p * lg2_approx(p + eps_log);
+    }
+    part[o] = tree8(v);
+  }
+  float S = tree<C::NOCT>(part);
+  if constexpr (C::LPT == 2) S = S + __shfl_xor_sync(kFull, S, 1);
+  return 0.0f - S;
+}
+
+// Exact score of one whole tile read straight from global memory by NOCT neighbouring lanes, lane o
+// taking the o-th group of eight elements (used for the few tiles near a group's threshold).  Same
+// arithmetic and summation tree as tile_score: the tree over the groups of eight runs as xor
+// shuffles (neighbours first; addition is commutative, so every lane ends with the same bits).
+// All 32 lanes of the warp must call it.
+template <int NOCT, bool BF16>
+__device__ __forceinline__ float exact_score_coop(const uint8_t *tile, int o, float eps_l1, float eps_log) {
+  float v[8];
+  if constexpr (BF16) {
+    const uint4 w = __ldg(reinterpret_cast<const uint4 *>(tile) + o);
+    const uint32_t u[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      v[2 * j] = __uint_as_float((u[j] << 16) & 0x7fffffffu);
+      v[2 * j + 1] = __uint_as_float(u[j] & 0x7fff0000u);
+    }
+  } else {
+    const float4 a = __ldg(reinterpret_cast<const float4 *>(tile) + 2 * o);
+    const float4 b = __ldg(reinterpret_cast<const float4 *>(tile) + 2 * o + 1);
+    v[0] = fabsf(a.x); v[1] = fabsf(a.y); v[2] = fabsf(a.z); v[3] = fabsf(a.w);
+    v[4] = fabsf(b.x); v[5] = fabsf(b.y); v[6] = fabsf(b.z); v[7] = fabsf(b.w);
+  }
+  float L1 = tree8(v);
+#pragma unroll
+  for (int h = 1; h < NOCT; h *= 2) L1 = L1 + __shfl_xor_sync(kFull, L1, h);
+  const float inv = __fdiv_rn(1.0f, L1 + eps_l1);
+#pragma unroll
+  for (int k = 0; k < 8; ++k) {
+    const float p = v[k] * inv;
+    v[k] = p * lg2_fma(p + eps_log);
+  }
+  float S = tree8(v);
+#pragma unroll
+  for (int h = 1; h < NOCT; h *= 2) S = S + __shfl_xor_sync(kFull, S, h);
   return 0.0f - S;
 }
 

@@ -13,6 +13,13 @@
 
 namespace tahq {
 
+#ifndef TAHQ_STATS_OCC
+#define TAHQ_STATS_OCC 2
+#endif
+#ifndef TAHQ_STATS_NST
+#define TAHQ_STATS_NST 2
+#endif
+
 struct Args {
   const uint8_t *in;        // encode: tensor; decode: unused
   uint8_t *packed;          // packed buffer (decode reads it)
@@ -25,6 +32,8 @@ struct Args {
   uint32_t *hist;           // [n_groups][kBins]   (zeroed per call)
   uint32_t *ncand;          // [n_groups]          (zeroed per call)
   uint32_t *done;           // [n_groups]          (zeroed per call) CTAs of select_kernel that finished a group
+  uint32_t *nabove;         // [n_groups]          (zeroed per call) tiles classified above the threshold band
+  uint32_t bf16, tile;      // element type and tile width of the tensor (select_kernel re-reads a few tiles)
   unsigned long long *theta;// [n_groups] ranking key of the k_hi-th ranked tile
   unsigned long long *cand; // [n_groups][cand_cap]
   uint32_t cand_cap, cpg;   // candidate capacity per group; CTAs per group of select_kernel
@@ -52,6 +61,17 @@ __device__ __forceinline__ void cta_chunk_range(uint64_t n_chunks, uint64_t &c0,
 template <class C, int NST, class Body>
 __device__ __forceinline__ void chunk_pipeline(const uint8_t *in, uint64_t n_tiles, uint64_t c0, uint64_t c1,
                                                uint8_t *stages, Body &&body) {
+  if constexpr (NST == 1) {   // no prefetch inside the CTA: several resident CTAs overlap each other instead
+    for (uint64_t c = c0; c < c1; ++c) {
+      issue_chunk<C>(in, n_tiles, c, stages);
+      cp_async_commit();
+      cp_async_wait<0>();
+      __syncthreads();
+      body(c, stages);
+      __syncthreads();
+    }
+    return;
+  }
   uint64_t c_issue = c0;
 #pragma unroll
   for (int s = 0; s < NST - 1; ++s) {
@@ -61,7 +81,7 @@ __device__ __forceinline__ void chunk_pipeline(const uint8_t *in, uint64_t n_til
   }
   int stage = 0;
   for (uint64_t c = c0; c < c1; ++c) {
-    cp_async_wait<NST - 2>();
+    cp_async_wait<(NST >= 2 ? NST - 2 : 0)>();
     __syncthreads();   // chunk c has landed; everyone is done with the stage consumed last time
     {
       const int s2 = (stage + NST - 1) % NST;
@@ -116,7 +136,7 @@ __device__ __forceinline__ uint64_t cta_exclusive_prefix(const Args &a, uint64_t
 // Eq. 1-2: entropy score per tile, plus the per-group histogram of binned scores (Sec. 3.2)
 // ------------------------------------------------------------------------------------------
 template <class C, int NST>
-__global__ void __launch_bounds__(kThreads) stats_kernel(const Args a) {
+__global__ void __launch_bounds__(kThreads, TAHQ_STATS_OCC) stats_kernel(const Args a) {
   extern __shared__ __align__(128) uint8_t smem[];
   __shared__ uint32_t s_hist[kBins];
   const bool use_hist = !a.direct;
@@ -138,7 +158,8 @@ __global__ void __launch_bounds__(kThreads) stats_kernel(const Args a) {
   cta_chunk_range(n_chunks, c0, c1);
   long long gcur = -1;
   chunk_pipeline<C, NST>(a.in, a.n_tiles, c0, c1, smem, [&](uint64_t c, const uint8_t *stage) {
-    const float s = tile_score<C>(stage, a.eps_l1, a.eps_log);
+    // small groups are ranked on exact scores; large ones are screened first (see select_kernel)
+    const float s = a.direct ? tile_score<C>(stage, a.eps_l1, a.eps_log) : tile_score_screen<C>(stage, a.eps_l1, a.eps_log);
     const uint64_t tile0 = c * C::TPC;
     const uint64_t tile = tile0 + threadIdx.x / C::LPT;
     const bool mine = tile < a.n_tiles && (C::LPT == 1 || !(threadIdx.x & 1));
@@ -172,10 +193,31 @@ template <class Get>
 __device__ __forceinline__ unsigned long long radix_select(uint64_t count, uint32_t r, Get &&get) {
   __shared__ uint32_t h[256];
   __shared__ uint32_t pick[2];
+  // bits on which the keys differ: a pass over a digit that is the same in every key is skipped
+  __shared__ unsigned long long s_or[kSelThreads / 32], s_and[kSelThreads / 32];
+  unsigned long long orv = 0, andv = ~0ull;
+  for (uint64_t i = threadIdx.x; i < count; i += kSelThreads) {
+    unsigned long long key;
+    if (get(i, key)) { orv |= key; andv &= key; }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    orv |= __shfl_xor_sync(kFull, orv, o);
+    andv &= __shfl_xor_sync(kFull, andv, o);
+  }
+  if ((threadIdx.x & 31) == 0) { s_or[threadIdx.x >> 5] = orv; s_and[threadIdx.x >> 5] = andv; }
+  __syncthreads();
+#pragma unroll
+  for (int w = 0; w < kSelThreads / 32; ++w) { orv |= s_or[w]; andv &= s_and[w]; }
+  const unsigned long long varying = orv ^ andv;
   unsigned long long prefix = 0, mask = 0;
   for (int shift = 56; shift >= 0; shift -= 8) {
+    if (((varying >> shift) & 0xffull) == 0) {   // every key has the same digit here
+      prefix |= orv & (0xffull << shift);
+      mask |= 0xffull << shift;
+      continue;
+    }
     if (threadIdx.x < 256) h[threadIdx.x] = 0;
-    __syncthreads();
     for (uint64_t i = threadIdx.x; i < count; i += kSelThreads) {
       unsigned long long key;
       if (get(i, key) && (key & mask) == prefix) atomicAdd(&h[(unsigned)(key >> shift) & 255u], 1u);
@@ -212,6 +254,10 @@ __device__ __forceinline__ unsigned long long radix_select(uint64_t count, uint3
 }
 
 constexpr int kSelSlice = 4 * kSelThreads;   // scores one CTA of select_kernel scans (four per thread, loaded at once)
+// Screening scores differ from exact ones by less than kScreenErr = 2.4e-4 (measured bound on the
+// approximate log2: 1e-5 per term, terms weighted by p with sum p <= 1, plus rounding); the band around
+// the threshold bin is 2*kScreenErr wide on each side, expressed in bins (kBinScale bins per unit).
+constexpr float kScreenBand = 0.25f;
 
 __global__ void __launch_bounds__(kSelThreads) select_kernel(const Args a) {
   extern __shared__ __align__(16) unsigned long long s_keys[];   // kSortCap keys
@@ -223,6 +269,12 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const Args a) {
   const float *sc = a.scores + g * ng;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   auto from_smem = [&](uint64_t i, unsigned long long &key) { key = s_keys[i]; return true; };
+#if defined(TAHQ_ABLATE) && (TAHQ_ABLATE & 16)
+  long long sk_t0 = clock64(), sk_prev = sk_t0; long long sk[6] = {0,0,0,0,0,0};
+#define SEL_TICK(i) do { long long n_ = clock64(); sk[i] += n_ - sk_prev; sk_prev = n_; } while (0)
+#else
+#define SEL_TICK(i) do {} while (0)
+#endif
 
   if (a.direct) {   // small group: rank all of its tiles here (one CTA per group)
     for (uint32_t i = threadIdx.x; i < (uint32_t)ng; i += kSelThreads) s_keys[i] = rank_key(sc[i], i);
@@ -267,49 +319,127 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const Args a) {
   }
   __syncthreads();
   const uint32_t B = s_sel[0], r = s_sel[1];
+  SEL_TICK(0);
 
-  // ---- B: candidates of bin B go to the group's list (one atomic per warp)
+  // ---- B: the scores so far are screening scores s~ (approximate log2), within kScreenErr of the
+  // exact ones, so the exact k_hi-th largest score lies within kScreenErr of bin B.  Tiles whose s~
+  // is more than 2*kScreenErr above (below) the bin are certainly inside (outside) the top k_hi: their
+  // score is replaced by +inf (-inf).  The rest are candidates: their exact score is recomputed from
+  // the tensor, stored, and ranked exactly in step C.
+  __shared__ uint32_t s_list[kSelSlice];
+  __shared__ uint32_t s_nlist, s_nabove;
+  if (threadIdx.x == 0) { s_nlist = 0; s_nabove = 0; }
+  __syncthreads();
+  float *scw = a.scores + g * ng;
+  const float band_lo = (float)B - kScreenBand, band_hi = (float)(B + 1) + kScreenBand;
 #pragma unroll
   for (int u = 0; u < 4; ++u) {
     const uint64_t i = lo + (uint64_t)u * kSelThreads + threadIdx.x;
-    const bool take = i < ng && score_bin(sv[u]) == B;
+    const float t = fmaxf(sv[u], 0.0f) * kBinScale;
+    const bool in = i < ng;
+    const bool above = in && t > band_hi, below = in && t < band_lo;
+    if (above) scw[i] = __int_as_float(0x7f800000);
+    if (below) scw[i] = __int_as_float(0xff800000);
+    const unsigned ma = __ballot_sync(kFull, above);
+    if (ma && lane == 0) atomicAdd(&s_nabove, (uint32_t)__popc(ma));
+    const bool take = in && !above && !below;
     const unsigned m = __ballot_sync(kFull, take);
     if (m) {
       uint32_t base = 0;
-      if (lane == 0) base = atomicAdd(&a.ncand[g], (uint32_t)__popc(m));
+      if (lane == 0) base = atomicAdd(&s_nlist, (uint32_t)__popc(m));
       base = __shfl_sync(kFull, base, 0);
-      const uint32_t slot = base + __popc(m & ((1u << lane) - 1u));
-      if (take && slot < a.cand_cap) a.cand[g * a.cand_cap + slot] = rank_key(sv[u], (uint32_t)i);
+      if (take) s_list[base + __popc(m & ((1u << lane) - 1u))] = (uint32_t)(i - lo);
+    }
+  }
+  __syncthreads();
+  SEL_TICK(1);
+  if (threadIdx.x == 0 && s_nabove) atomicAdd(&a.nabove[g], s_nabove);
+  {
+    const uint32_t nl = s_nlist;
+    const uint32_t tile_bytes = a.tile * (a.bf16 ? 2u : 4u);
+    uint32_t slot0 = 0;
+    __shared__ uint32_t s_slot0;
+    if (threadIdx.x == 0) s_slot0 = atomicAdd(&a.ncand[g], nl);
+    __syncthreads();
+    slot0 = s_slot0;
+    // candidates, densely over the threads: NOCT = tile/8 neighbouring lanes share one candidate
+    const uint32_t noct = a.tile / 8, per_round = kSelThreads / noct;
+    const uint32_t sub = threadIdx.x % noct;
+    for (uint32_t j0 = 0; j0 < nl; j0 += per_round) {   // uniform trip count: whole warps take part
+      const uint32_t j = j0 + threadIdx.x / noct;
+      const bool live = j < nl;
+      const uint64_t i = lo + s_list[live ? j : 0];
+      const uint8_t *tp = a.in + (g * ng + i) * (uint64_t)tile_bytes;
+      float ex;
+      if (a.bf16) {
+        ex = noct == 4   ? exact_score_coop<4, true>(tp, sub, a.eps_l1, a.eps_log)
+             : noct == 8 ? exact_score_coop<8, true>(tp, sub, a.eps_l1, a.eps_log)
+                         : exact_score_coop<16, true>(tp, sub, a.eps_l1, a.eps_log);
+      } else {
+        ex = noct == 4   ? exact_score_coop<4, false>(tp, sub, a.eps_l1, a.eps_log)
+             : noct == 8 ? exact_score_coop<8, false>(tp, sub, a.eps_l1, a.eps_log)
+                         : exact_score_coop<16, false>(tp, sub, a.eps_l1, a.eps_log);
+      }
+      if (live && sub == 0) {
+        scw[i] = ex;
+        if (slot0 + j < a.cand_cap) a.cand[g * a.cand_cap + slot0 + j] = rank_key(ex, (uint32_t)i);
+      }
     }
   }
 
+  SEL_TICK(2);
   // ---- C: the CTA that finishes the group last ranks the candidates exactly
   __threadfence();
   __syncthreads();
   if (threadIdx.x == 0) s_last = atomicAdd(&a.done[g], 1u) == a.cpg - 1;
   __syncthreads();
+#if defined(TAHQ_ABLATE) && (TAHQ_ABLATE & 16)
+  SEL_TICK(3);
+  if (threadIdx.x == 0) { for (int i = 0; i < 4; ++i) a.flags[256 + blockIdx.x * 8 + i] = (unsigned long long)sk[i]; a.flags[256 + blockIdx.x * 8 + 6] = s_nlist; }
+#endif
   if (!s_last) return;
   __threadfence();
-  const uint32_t n = gh[B];
+  const uint32_t n = *reinterpret_cast<volatile uint32_t *>(a.ncand + g);
+  const uint32_t nab = *reinterpret_cast<volatile uint32_t *>(a.nabove + g);
+  uint32_t rr = (uint32_t)a.k_hi - nab;   // rank of the threshold tile among the candidates
+  if (nab >= (uint32_t)a.k_hi || rr > n) {   // only possible if the screening error exceeded its bound
+    if (threadIdx.x == 0) atomicOr(a.status, 8u /* TAHQ_DEV_INTERNAL */);
+    rr = rr > n ? n : 1u;
+    if (n == 0) { if (threadIdx.x == 0) a.theta[g] = ~0ull; return; }
+  }
+  (void)r;
   const unsigned long long *cand = a.cand + g * a.cand_cap;
   unsigned long long t;
-  if (n <= a.cand_cap && n <= (uint32_t)kSortCap) {
+  if (n <= a.cand_cap && n <= (uint32_t)kSelThreads) {
+    // few candidates (the usual case): every thread ranks one key by counting the larger ones
+    const unsigned long long mine = threadIdx.x < n ? __ldcg(cand + threadIdx.x) : 0ull;
+    s_keys[threadIdx.x] = mine;
+    __syncthreads();
+    uint32_t larger = 0;
+    for (uint32_t i = 0; i < n; ++i) larger += s_keys[i] > mine ? 1u : 0u;
+    if (threadIdx.x < n && larger == rr - 1) a.theta[g] = mine;   // keys are distinct: exactly one thread
+    return;
+  } else if (n <= a.cand_cap && n <= (uint32_t)kSortCap) {
     for (uint32_t i = threadIdx.x; i < n; i += kSelThreads) s_keys[i] = __ldcg(cand + i);
     __syncthreads();
-    t = radix_select(n, r, from_smem);
+    t = radix_select(n, rr, from_smem);
   } else if (n <= a.cand_cap) {
-    t = radix_select(n, r, [&](uint64_t i, unsigned long long &key) {
+    t = radix_select(n, rr, [&](uint64_t i, unsigned long long &key) {
       key = __ldcg(cand + i);
       return true;
     });
-  } else {   // more candidates than the list holds: take them from the scores
-    t = radix_select(ng, r, [&](uint64_t i, unsigned long long &key) {
-      const float s = sc[i];
+  } else {   // more candidates than the list holds: they are exactly the tiles whose stored score is finite
+    t = radix_select(ng, rr, [&](uint64_t i, unsigned long long &key) {
+      const float s = __ldcg(scw + i);
       key = rank_key(s, (uint32_t)i);
-      return score_bin(s) == B;
+      return (__float_as_uint(s) & 0x7f800000u) != 0x7f800000u;
     });
   }
   if (threadIdx.x == 0) a.theta[g] = t;
+#if defined(TAHQ_ABLATE) && (TAHQ_ABLATE & 16)
+  SEL_TICK(4);
+  if (threadIdx.x == 0) { a.flags[256 + blockIdx.x * 8 + 4] = (unsigned long long)sk[4]; a.flags[256 + blockIdx.x * 8 + 5] = n; }
+#endif
 }
 
 // Is tile `tile` one of the k_hi highest-ranked tiles of its group?
