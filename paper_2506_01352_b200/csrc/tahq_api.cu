@@ -217,7 +217,7 @@ static tahq_status encode_t(const Plan &pl, const Args &a, cudaStream_t st) {
     TAHQ_LAUNCH("select", st, select_kernel<<<(unsigned)(a.n_groups * a.cpg), kSelThreads, sel_smem, st>>>(a));
   }
   constexpr int NQ = Stages<C>::QUANT;
-  const int smem = NQ * C::STAGE_BYTES;
+  const int smem = NQ * (C::STAGE_BYTES + C::TPC * 4);
   const int occ = prepare(quant_pack_kernel<C, NQ>, smem, d, occ_quant);
   if (!occ) return TAHQ_ERR_CUDA;
   TAHQ_LAUNCH("quant_pack", st,

@@ -98,8 +98,14 @@ __device__ __forceinline__ bool mbar_wait(unsigned long long *bar, unsigned pari
 // Copy the rows of chunk `c` (tiles [c*TPC, (c+1)*TPC), clipped to n_tiles) into a swizzled stage.
 // Rows past the end of the tensor are zero-filled.
 template <class C>
-__device__ __forceinline__ void issue_chunk(const uint8_t *in, uint64_t n_tiles, uint64_t c, uint8_t *stage) {
+__device__ __forceinline__ void issue_chunk(const uint8_t *in, uint64_t n_tiles, uint64_t c, uint8_t *stage,
+                                            const float *scores = nullptr) {
   const uint64_t tile0 = c * C::TPC;
+  if (scores && threadIdx.x < C::TPC / 4) {   // the chunk's scores ride along behind the rows
+    const uint64_t first = tile0 + (uint64_t)threadIdx.x * 4;
+    const int left = first < n_tiles ? (int)(n_tiles - first < 4 ? n_tiles - first : 4) : 0;
+    cp_async16(stage + C::STAGE_BYTES + (size_t)threadIdx.x * 16, left ? scores + first : scores, left * 4);
+  }
   const uint8_t *src = in + tile0 * (uint64_t)(C::G * C::ESZ) + (size_t)threadIdx.x * 16;
   // chunk index ci = i*kThreads + tid lies in row ci / CPR, whose swizzle depends on tid only
   uint8_t *dst = stage + (size_t)((int)threadIdx.x ^ swz<C>((int)threadIdx.x / C::CPR)) * 16;
@@ -609,6 +615,43 @@ __device__ __forceinline__ ClassSort sort_by_class(int cls, uint8_t *s_perm, uin
   const int t = threadIdx.x;
   r.cls = (t >= base1) + (t >= base2) + (t >= base3);
   return r;
+}
+
+// Smallest and largest element of a row.
+template <class C>
+__device__ __forceinline__ void row_minmax(const uint8_t *stage, int row, float &mn, float &mx) {
+  if constexpr (C::BF16) {
+    uint32_t lo0, lo1, hi0, hi1;
+#pragma unroll
+    for (int q = 0; q < C::CPR; ++q) {
+      const uint4 w = *reinterpret_cast<const uint4 *>(stage + (size_t)phys_chunk<C>(row, q) * 16);
+      if (q == 0) {
+        lo0 = bf2_min(w.x, w.z); hi0 = bf2_max(w.x, w.z);
+        lo1 = bf2_min(w.y, w.w); hi1 = bf2_max(w.y, w.w);
+      } else {
+        lo0 = bf2_min(lo0, bf2_min(w.x, w.z)); hi0 = bf2_max(hi0, bf2_max(w.x, w.z));
+        lo1 = bf2_min(lo1, bf2_min(w.y, w.w)); hi1 = bf2_max(hi1, bf2_max(w.y, w.w));
+      }
+    }
+    lo0 = bf2_min(lo0, lo1); hi0 = bf2_max(hi0, hi1);
+    mn = fminf(__uint_as_float(lo0 << 16), __uint_as_float(lo0 & 0xffff0000u));
+    mx = fmaxf(__uint_as_float(hi0 << 16), __uint_as_float(hi0 & 0xffff0000u));
+  } else {
+    float l0, l1, h0, h1;
+#pragma unroll
+    for (int q = 0; q < C::CPR; ++q) {
+      const float4 v = *reinterpret_cast<const float4 *>(stage + (size_t)phys_chunk<C>(row, q) * 16);
+      if (q == 0) {
+        l0 = fminf(v.x, v.z); h0 = fmaxf(v.x, v.z);
+        l1 = fminf(v.y, v.w); h1 = fmaxf(v.y, v.w);
+      } else {
+        l0 = fminf(l0, fminf(v.x, v.z)); h0 = fmaxf(h0, fmaxf(v.x, v.z));
+        l1 = fminf(l1, fminf(v.y, v.w)); h1 = fmaxf(h1, fmaxf(v.y, v.w));
+      }
+    }
+    mn = fminf(l0, l1);
+    mx = fmaxf(h0, h1);
+  }
 }
 
 // Largest and second-largest magnitude of a row (Eq. 3), no index.

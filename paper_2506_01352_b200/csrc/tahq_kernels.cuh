@@ -60,10 +60,12 @@ __device__ __forceinline__ void cta_chunk_range(uint64_t n_chunks, uint64_t &c0,
 // ------------------------------------------------------------------------------------------
 template <class C, int NST, class Body>
 __device__ __forceinline__ void chunk_pipeline(const uint8_t *in, uint64_t n_tiles, uint64_t c0, uint64_t c1,
-                                               uint8_t *stages, Body &&body) {
+                                               uint8_t *stages, Body &&body, const float *scores = nullptr) {
+  // a stage holds the chunk's rows and, when `scores` is given, the chunk's TPC scores behind them
+  const size_t stride = (size_t)C::STAGE_BYTES + (scores ? (size_t)C::TPC * 4 : 0);
   if constexpr (NST == 1) {   // no prefetch inside the CTA: several resident CTAs overlap each other instead
     for (uint64_t c = c0; c < c1; ++c) {
-      issue_chunk<C>(in, n_tiles, c, stages);
+      issue_chunk<C>(in, n_tiles, c, stages, scores);
       cp_async_commit();
       cp_async_wait<0>();
       __syncthreads();
@@ -75,7 +77,7 @@ __device__ __forceinline__ void chunk_pipeline(const uint8_t *in, uint64_t n_til
   uint64_t c_issue = c0;
 #pragma unroll
   for (int s = 0; s < NST - 1; ++s) {
-    if (c_issue < c1) issue_chunk<C>(in, n_tiles, c_issue, stages + (size_t)s * C::STAGE_BYTES);
+    if (c_issue < c1) issue_chunk<C>(in, n_tiles, c_issue, stages + (size_t)s * stride, scores);
     cp_async_commit();
     ++c_issue;
   }
@@ -85,11 +87,11 @@ __device__ __forceinline__ void chunk_pipeline(const uint8_t *in, uint64_t n_til
     __syncthreads();   // chunk c has landed; everyone is done with the stage consumed last time
     {
       const int s2 = (stage + NST - 1) % NST;
-      if (c_issue < c1) issue_chunk<C>(in, n_tiles, c_issue, stages + (size_t)s2 * C::STAGE_BYTES);
+      if (c_issue < c1) issue_chunk<C>(in, n_tiles, c_issue, stages + (size_t)s2 * stride, scores);
       cp_async_commit();
       ++c_issue;
     }
-    body(c, stages + (size_t)stage * C::STAGE_BYTES);
+    body(c, stages + (size_t)stage * stride);
     stage = (stage + 1) % NST;
   }
   cp_async_wait<0>();
@@ -159,7 +161,11 @@ __global__ void __launch_bounds__(kThreads, TAHQ_STATS_OCC) stats_kernel(const A
   long long gcur = -1;
   chunk_pipeline<C, NST>(a.in, a.n_tiles, c0, c1, smem, [&](uint64_t c, const uint8_t *stage) {
     // small groups are ranked on exact scores; large ones are screened first (see select_kernel)
+#if defined(TAHQ_ABLATE) && (TAHQ_ABLATE & 32)
+    const float s = *reinterpret_cast<const float *>(stage + threadIdx.x * 16);
+#else
     const float s = a.direct ? tile_score<C>(stage, a.eps_l1, a.eps_log) : tile_score_screen<C>(stage, a.eps_l1, a.eps_log);
+#endif
     const uint64_t tile0 = c * C::TPC;
     const uint64_t tile = tile0 + threadIdx.x / C::LPT;
     const bool mine = tile < a.n_tiles && (C::LPT == 1 || !(threadIdx.x & 1));
@@ -473,6 +479,13 @@ struct GroupCursor {
     if (i >= a.tiles_per_group) { gg += i / a.tiles_per_group; i %= a.tiles_per_group; }
     return rank_key(__ldg(a.scores + tile), (uint32_t)i) >= __ldg(a.theta + gg);
   }
+  // the same with the tile's score already at hand
+  __device__ __forceinline__ bool is_hi_score(const Args &a, float score, uint32_t off) const {
+    uint64_t gg = g;
+    uint64_t i = (uint64_t)rem + off;
+    if (i >= a.tiles_per_group) { gg += i / a.tiles_per_group; i %= a.tiles_per_group; }
+    return rank_key(score, (uint32_t)i) >= __ldg(a.theta + gg);
+  }
 };
 
 __device__ __forceinline__ uint32_t block_sum(uint32_t v) {
@@ -654,23 +667,14 @@ __device__ __forceinline__ void quantise_pairs(float2 (&p)[NPAIR], float mn, flo
 // Unflagged bf16 rows never need their elements widened one by one: min/max run on the packed
 // words, and the quantiser's first operation takes the bf16 half as an operand.
 template <class C>
-__device__ __forceinline__ Quantiser encode_raw_bf16_row(const uint8_t *stage, int row, uint32_t bits, uint32_t *dst,
-                                                          bool store) {
+__device__ __forceinline__ Quantiser encode_raw_bf16_row(const uint8_t *stage, int row, float mn, float mx,
+                                                          uint32_t bits, uint32_t *dst, bool store) {
   uint32_t w[C::EPT / 2];
 #pragma unroll
   for (int q = 0; q < C::CPR; ++q) {
     const uint4 v = *reinterpret_cast<const uint4 *>(stage + (size_t)phys_chunk<C>(row, q) * 16);
     w[4 * q] = v.x; w[4 * q + 1] = v.y; w[4 * q + 2] = v.z; w[4 * q + 3] = v.w;
   }
-  uint32_t lo0 = w[0], lo1 = w[1], hi0 = w[0], hi1 = w[1];
-#pragma unroll
-  for (int j = 2; j < C::EPT / 2; j += 2) {
-    lo0 = bf2_min(lo0, w[j]); hi0 = bf2_max(hi0, w[j]);
-    lo1 = bf2_min(lo1, w[j + 1]); hi1 = bf2_max(hi1, w[j + 1]);
-  }
-  lo0 = bf2_min(lo0, lo1); hi0 = bf2_max(hi0, hi1);
-  const float mn = fminf(__uint_as_float(lo0 << 16), __uint_as_float(lo0 & 0xffff0000u));
-  const float mx = fmaxf(__uint_as_float(hi0 << 16), __uint_as_float(hi0 & 0xffff0000u));
   const Quantiser q = make_quantiser(mn, mx, bits);
   const float ymin = (mn - q.z) * q.inv_s, ymax = (mx - q.z) * q.inv_s;
   const bool safe = ymin >= -0.4999f && ymax < q.qmax + 0.4999f;
@@ -701,7 +705,7 @@ __global__ void __launch_bounds__(kThreads, 2) quant_pack_kernel(const Args a) {
   __shared__ uint8_t s_perm[kThreads];
   __shared__ uint2 s_cnt[kThreads / 32];
   __shared__ uint16_t s_rowoff[kThreads];
-  __shared__ float s_a1[kThreads];
+  __shared__ float2 s_mnmx[kThreads];
   uint32_t *sz32 = reinterpret_cast<uint32_t *>(a.packed + a.off_sz);
   uint8_t *pivot = a.packed + a.off_pivot;
   uint32_t *bitmap = reinterpret_cast<uint32_t *>(a.packed + a.off_bitmap);
@@ -742,36 +746,48 @@ __global__ void __launch_bounds__(kThreads, 2) quant_pack_kernel(const Args a) {
     const uint64_t left = a.n_tiles - tile0;
     const uint32_t nvalid = left < (uint64_t)C::TPC ? (uint32_t)left : (uint32_t)C::TPC;
     const uint32_t own = threadIdx.x / C::LPT;   // tile of the chunk this thread looks at first
-    const bool hi1 = a.mixed && own < nvalid && cur.is_hi(a, tile0 + own, own);
+    const float *sc_stage = reinterpret_cast<const float *>(stage + C::STAGE_BYTES);   // staged with the rows
+    const bool hi1 = a.mixed && own < nvalid && cur.is_hi_score(a, sc_stage[own], own);
     const uint64_t goff = (uint64_t)(C::G / 8) * ((uint64_t)a.lo * tile0 + hi_run);
 
     if constexpr (C::LPT == 1) {
-      // ---- phase 1: thread r looks at tile r: outlier test (Eq. 3), then the CTA regroups its tiles
-      float a1, a2;
-      row_top2<C>(stage, (int)threadIdx.x, a1, a2);
-      const float t1 = a2 + a.eps_ratio;
-      const float t2 = a.tau * t1;
-      const bool flag1 = a1 > t2;
-      const Regroup rg = regroup((flag1 ? 2 : 0) | (hi1 ? 1 : 0), s_perm, s_cnt, [&](const Regroup &r) {
+      // ---- phase 1: thread r looks at tile r: range of the row, and a first look at Eq. 3.  The second-
+      // largest magnitude is at least the smaller of |min| and |max| (they sit at different positions,
+      // or every element is equal), so a tile whose largest magnitude does not exceed
+      // tau * (that + varrho) cannot be flagged; only the others ("maybe") need the exact top two.
+      float mn1, mx1;
+      row_minmax<C>(stage, (int)threadIdx.x, mn1, mx1);
+      const float m_big = fmaxf(fabsf(mn1), fabsf(mx1)), m_small = fminf(fabsf(mn1), fabsf(mx1));
+      const bool maybe1 = m_big > a.tau * (m_small + a.eps_ratio);
+      const Regroup rg = regroup((maybe1 ? 2 : 0) | (hi1 ? 1 : 0), s_perm, s_cnt, [&](const Regroup &r) {
         s_rowoff[threadIdx.x] = (uint16_t)((C::G / 8) * (a.lo * threadIdx.x + r.hi_before));
-        s_a1[threadIdx.x] = a1;
+        s_mnmx[threadIdx.x] = make_float2(mn1, mx1);
         if ((threadIdx.x & 31) == 0) bitmap[tile0 / 32 + (threadIdx.x >> 5)] = r.hi_ballot;
       });
       hi_run += rg.total_hi;
       // ---- phase 2: this thread now owns tile `src` of the chunk
       const int src = rg.src;
-      const bool flag = rg.cls & 2;
+      const bool maybe = rg.cls & 2;
       const uint32_t b = a.lo + (rg.cls & 1);
       const uint64_t tile = tile0 + src;
       const bool live = (uint32_t)src < nvalid;
       uint32_t *dst = reinterpret_cast<uint32_t *>(a.packed + a.off_payload + goff + s_rowoff[src]);
-      if (C::BF16 && !flag) {
-        const Quantiser q = encode_raw_bf16_row<C>(stage, src, b, dst, live);
+      if (C::BF16 && !maybe) {
+        const float2 mm = s_mnmx[src];
+        const Quantiser q = encode_raw_bf16_row<C>(stage, src, mm.x, mm.y, b, dst, live);
         if (live) { sz32[tile] = q.sz; pivot[tile] = 0; }
       } else {
+        float a1 = 0.0f, a2 = 0.0f;
+        bool flag = false;
+        if (maybe) {   // Eq. 3 exactly
+          row_top2<C>(stage, src, a1, a2);
+          const float t1 = a2 + a.eps_ratio;
+          const float t2 = a.tau * t1;
+          flag = a1 > t2;
+        }
         int d = 0;
         if (flag) {   // Eq. 4: the pivot swap P_d, done in place in shared memory before the row is loaded
-          d = row_first_index_of<C>(stage, src, s_a1[src]);
+          d = row_first_index_of<C>(stage, src, a1);
           row_swap_0_d<C, !C::BF16>(const_cast<uint8_t *>(stage), src, d);
           asm volatile("" ::: "memory");
         }
@@ -875,7 +891,7 @@ __global__ void __launch_bounds__(kThreads, 2) quant_pack_kernel(const Args a) {
       }
     }
     cur.advance(a, C::TPC);
-  });
+  }, a.mixed ? a.scores : nullptr);
 }
 
 // ------------------------------------------------------------------------------------------
