@@ -6,7 +6,7 @@
 #include <cstring>
 #include <vector>
 
-#include "tahq_kernels.cuh"
+#include "tahq_stream.cuh"
 
 namespace tahq {
 
@@ -185,7 +185,7 @@ static int prepare(K kernel, int smem, const DevInfo &d, std::atomic<int> *cache
 }
 
 template <class C> struct Stages {
-  static constexpr int STATS = (C::ROWB == 256) ? 2 : TAHQ_STATS_NST;
+  static constexpr int STATS = 2;
   static constexpr int QUANT = (C::ROWB == 256) ? 2 : (C::ROWB == 128 ? 2 : 3);
 };
 
@@ -216,12 +216,23 @@ static tahq_status encode_t(const Plan &pl, const Args &a, cudaStream_t st) {
     }
     TAHQ_LAUNCH("select", st, select_kernel<<<(unsigned)(a.n_groups * a.cpg), kSelThreads, sel_smem, st>>>(a));
   }
-  constexpr int NQ = Stages<C>::QUANT;
-  const int smem = NQ * (C::STAGE_BYTES + C::TPC * 4);
-  const int occ = prepare(quant_pack_kernel<C, NQ>, smem, d, occ_quant);
-  if (!occ) return TAHQ_ERR_CUDA;
-  TAHQ_LAUNCH("quant_pack", st,
-              quant_pack_kernel<C, NQ><<<persistent_grid(n_chunks, d, occ), kThreads, smem, st>>>(a));
+  if constexpr (C::LPT == 1) {   // one lane per tile: warps stream units of 32 tiles independently
+    constexpr int NQ = 2;
+    const int smem = StreamCfg<C>::smem_bytes(NQ);
+    const int occ = prepare(quant_pack_stream_kernel<C, NQ>, smem, d, occ_quant);
+    if (!occ) return TAHQ_ERR_CUDA;
+    const uint64_t n_units = (a.n_tiles + 31) / 32;
+    TAHQ_LAUNCH("quant_pack", st,
+                quant_pack_stream_kernel<C, NQ><<<persistent_grid((n_units + kWarps - 1) / kWarps, d, occ), kThreads,
+                                                  smem, st>>>(a));
+  } else {
+    constexpr int NQ = Stages<C>::QUANT;
+    const int smem = NQ * (C::STAGE_BYTES + C::TPC * 4);
+    const int occ = prepare(quant_pack_kernel<C, NQ>, smem, d, occ_quant);
+    if (!occ) return TAHQ_ERR_CUDA;
+    TAHQ_LAUNCH("quant_pack", st,
+                quant_pack_kernel<C, NQ><<<persistent_grid(n_chunks, d, occ), kThreads, smem, st>>>(a));
+  }
   return cudaGetLastError() == cudaSuccess ? TAHQ_OK : TAHQ_ERR_CUDA;
 }
 

@@ -231,58 +231,13 @@ __device__ __forceinline__ float2 fma2(float2 a, float2 b, float2 c) {
   return d;
 }
 
-// log2 of positive normal numbers: exponent + u*Q(u), u = mantissa - 1, Q of degree 5.
-__device__ __forceinline__ float2 lg2_poly2(float2 x) {
-  const uint32_t x0 = __float_as_uint(x.x), x1 = __float_as_uint(x.y);
-  const float2 e = add2(f2((float)(int)(x0 >> 23), (float)(int)(x1 >> 23)), f2(-127.0f));
-  const float2 m = f2(__uint_as_float((x0 & 0x007fffffu) | 0x3f800000u), __uint_as_float((x1 & 0x007fffffu) | 0x3f800000u));
-  const float2 u = add2(m, f2(-1.0f));
-  float2 q = f2(-0x1.a762d6p-6f);
-  q = fma2(q, u, f2(0x1.f2e252p-4f));
-  q = fma2(q, u, f2(-0x1.1c9334p-2f));
-  q = fma2(q, u, f2(0x1.d487c6p-2f));
-  q = fma2(q, u, f2(-0x1.6fb0bcp-1f));
-  q = fma2(q, u, f2(0x1.714aa0p+0f));
-  return fma2(u, q, e);
-}
-
-// neighbours-first pairwise tree over 8 pairs (each lane of the pair is its own sum)
-__device__ __forceinline__ float2 tree8x2(const float2 (&v)[8]) {
-  const float2 a = add2(v[0], v[1]), b = add2(v[2], v[3]);
-  const float2 c = add2(v[4], v[5]), d = add2(v[6], v[7]);
-  return add2(add2(a, b), add2(c, d));
-}
-
-// Magnitudes of octs 2p and 2p+1 of a row, element k of both octs in one pair.
-template <class C>
-__device__ __forceinline__ void load_abs_oct_pair(const uint8_t *stage, int row, int p, float2 (&a)[8]) {
-  if constexpr (C::BF16) {
-    const uint4 w0 = *reinterpret_cast<const uint4 *>(stage + (size_t)phys_chunk<C>(row, 2 * p) * 16);
-    const uint4 w1 = *reinterpret_cast<const uint4 *>(stage + (size_t)phys_chunk<C>(row, 2 * p + 1) * 16);
-    const uint32_t u0[4] = {w0.x, w0.y, w0.z, w0.w}, u1[4] = {w1.x, w1.y, w1.z, w1.w};
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      float l0, h0, l1, h1;   // clearing the sign bits of the packed word, then widening on the FMA pipe
-      bf2_add_f32(u0[j] & 0x7fff7fffu, -0.0f, l0, h0);
-      bf2_add_f32(u1[j] & 0x7fff7fffu, -0.0f, l1, h1);
-      a[2 * j] = f2(l0, l1);
-      a[2 * j + 1] = f2(h0, h1);
-    }
-  } else {
-    float v0[8], v1[8];
-    load_oct<C>(stage, row, 2 * p, v0);
-    load_oct<C>(stage, row, 2 * p + 1, v1);
-#pragma unroll
-    for (int k = 0; k < 8; ++k) a[k] = f2(fabsf(v0[k]), fabsf(v1[k]));
-  }
-}
-
-// log2 of a positive normal number, exponent + u*Q(u) as in lg2_poly, with the exponent and the
+// log2 of a positive normal number as exponent + u*Q(u) (u = mantissa - 1, Q a fixed degree-5
+// polynomial evaluated by Horner's rule with fused multiply-adds), with the exponent and the
 // mantissa split done by multiply-adds so that everything runs on the FMA pipe (the ALU pipe has
 // half its rate and is the busier one):  (x * 512) >> 32 is the biased exponent eb, placed into the
 // mantissa of 2^23 by the addend of the same integer multiply-add; 2^-E is built as a bit pattern
-// by one more integer multiply-add, and u = x * 2^-E - 1 is exact (so is every step: the result has
-// the same bits as lg2_poly).
+// by one more integer multiply-add, and u = x * 2^-E - 1 is exact, as is every step before the
+// polynomial.
 __device__ __forceinline__ float lg2_fma(float x) {
   const uint32_t xi = __float_as_uint(x);
   uint32_t ebm;
@@ -453,22 +408,6 @@ __device__ __forceinline__ void butterfly(float (&x)[N]) {
       }
 }
 
-template <class C>
-__device__ __forceinline__ void hadamard_scaled(float (&x)[C::EPT]) {
-  butterfly<C::EPT>(x);
-  if constexpr (C::LPT == 2) {
-    const bool upper = threadIdx.x & 1;
-#pragma unroll
-    for (int k = 0; k < C::EPT; ++k) {
-      const float p = __shfl_xor_sync(kFull, x[k], 1);
-      x[k] = upper ? (p - x[k]) : (x[k] + p);
-    }
-  }
-  constexpr float c = (C::G == 32) ? 0.17677669529663687f : (C::G == 64) ? 0.125f : 0.08838834764831845f;
-#pragma unroll
-  for (int k = 0; k < C::EPT; ++k) x[k] = x[k] * c;
-}
-
 // The same butterfly on adjacent pairs p[i] = (x[2i], x[2i+1]): stride 1 works inside a pair, every
 // larger stride adds and subtracts whole pairs (a - b is formed as fma(b, -1, a), which is exact).
 template <int NPAIR>
@@ -557,29 +496,6 @@ __device__ __forceinline__ void row_swap_0_d(uint8_t *stage, int row, int d) {
   }
 }
 
-// Little-endian bit stream of N codes of W bits into N*W/32 words (all indices static).
-template <int W, int N>
-__device__ __forceinline__ void pack_words(const uint32_t (&c)[N], uint32_t *w) {
-#pragma unroll
-  for (int j = 0; j < N * W / 32; ++j) w[j] = 0;
-#pragma unroll
-  for (int k = 0; k < N; ++k) {
-    const int bit = k * W, j = bit >> 5, s = bit & 31;
-    w[j] |= c[k] << s;
-    if (s + W > 32) w[j + 1] |= c[k] >> (32 - s);
-  }
-}
-template <int W, int N>
-__device__ __forceinline__ void unpack_words(const uint32_t *w, uint32_t (&c)[N]) {
-#pragma unroll
-  for (int k = 0; k < N; ++k) {
-    const int bit = k * W, j = bit >> 5, s = bit & 31;
-    uint32_t v = w[j] >> s;
-    if (s + W > 32) v |= w[j + 1] << (32 - s);
-    c[k] = v & ((1u << W) - 1u);
-  }
-}
-
 // ------------------------------------------------------------------------------------------
 // Stable counting sort of the 256 threads of a CTA by a 2-bit class, so that the warps that go
 // on are (nearly) uniform in (transformed?, higher width?) and neither the Hadamard butterfly nor
@@ -589,71 +505,6 @@ struct ClassSort {
   int src;   // which thread's tile this thread processes from now on
   int cls;   // class of that tile
 };
-__device__ __forceinline__ ClassSort sort_by_class(int cls, uint8_t *s_perm, uint2 *s_cnt) {
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const unsigned b1 = __ballot_sync(kFull, cls & 1), b2 = __ballot_sync(kFull, cls & 2);
-  const unsigned m0 = ~b1 & ~b2, m1 = b1 & ~b2, m2 = ~b1 & b2, m3 = b1 & b2;
-  if (lane == 0) s_cnt[warp] = make_uint2(__popc(m0) | (__popc(m1) << 16), __popc(m2) | (__popc(m3) << 16));
-  __syncthreads();
-  uint32_t tot_lo = 0, tot_hi = 0, bef_lo = 0, bef_hi = 0;   // two 16-bit counters per word
-#pragma unroll
-  for (int w = 0; w < kThreads / 32; ++w) {
-    const uint2 c = s_cnt[w];
-    tot_lo += c.x; tot_hi += c.y;
-    bef_lo += (w < warp) ? c.x : 0u;
-    bef_hi += (w < warp) ? c.y : 0u;
-  }
-  const int base1 = tot_lo & 0xffff, base2 = base1 + (tot_lo >> 16), base3 = base2 + (tot_hi & 0xffff);
-  const unsigned mine = (cls == 0) ? m0 : (cls == 1) ? m1 : (cls == 2) ? m2 : m3;
-  const int before = (cls == 0) ? (bef_lo & 0xffff) : (cls == 1) ? (bef_lo >> 16) : (cls == 2) ? (bef_hi & 0xffff)
-                                                                                               : (bef_hi >> 16);
-  const int base = (cls == 0) ? 0 : (cls == 1) ? base1 : (cls == 2) ? base2 : base3;
-  s_perm[base + before + __popc(mine & ((1u << lane) - 1u))] = (uint8_t)threadIdx.x;
-  __syncthreads();
-  ClassSort r;
-  r.src = s_perm[threadIdx.x];
-  const int t = threadIdx.x;
-  r.cls = (t >= base1) + (t >= base2) + (t >= base3);
-  return r;
-}
-
-// Smallest and largest element of a row.
-template <class C>
-__device__ __forceinline__ void row_minmax(const uint8_t *stage, int row, float &mn, float &mx) {
-  if constexpr (C::BF16) {
-    uint32_t lo0, lo1, hi0, hi1;
-#pragma unroll
-    for (int q = 0; q < C::CPR; ++q) {
-      const uint4 w = *reinterpret_cast<const uint4 *>(stage + (size_t)phys_chunk<C>(row, q) * 16);
-      if (q == 0) {
-        lo0 = bf2_min(w.x, w.z); hi0 = bf2_max(w.x, w.z);
-        lo1 = bf2_min(w.y, w.w); hi1 = bf2_max(w.y, w.w);
-      } else {
-        lo0 = bf2_min(lo0, bf2_min(w.x, w.z)); hi0 = bf2_max(hi0, bf2_max(w.x, w.z));
-        lo1 = bf2_min(lo1, bf2_min(w.y, w.w)); hi1 = bf2_max(hi1, bf2_max(w.y, w.w));
-      }
-    }
-    lo0 = bf2_min(lo0, lo1); hi0 = bf2_max(hi0, hi1);
-    mn = fminf(__uint_as_float(lo0 << 16), __uint_as_float(lo0 & 0xffff0000u));
-    mx = fmaxf(__uint_as_float(hi0 << 16), __uint_as_float(hi0 & 0xffff0000u));
-  } else {
-    float l0, l1, h0, h1;
-#pragma unroll
-    for (int q = 0; q < C::CPR; ++q) {
-      const float4 v = *reinterpret_cast<const float4 *>(stage + (size_t)phys_chunk<C>(row, q) * 16);
-      if (q == 0) {
-        l0 = fminf(v.x, v.z); h0 = fmaxf(v.x, v.z);
-        l1 = fminf(v.y, v.w); h1 = fmaxf(v.y, v.w);
-      } else {
-        l0 = fminf(l0, fminf(v.x, v.z)); h0 = fmaxf(h0, fmaxf(v.x, v.z));
-        l1 = fminf(l1, fminf(v.y, v.w)); h1 = fmaxf(h1, fmaxf(v.y, v.w));
-      }
-    }
-    mn = fminf(l0, l1);
-    mx = fmaxf(h0, h1);
-  }
-}
-
 // Largest and second-largest magnitude of a row (Eq. 3), no index.
 template <class C>
 __device__ __forceinline__ void row_top2(const uint8_t *stage, int row, float &a1, float &a2) {

@@ -3,7 +3,9 @@
 //   encode:  stats_kernel        Eq. 1-2   tile -> entropy score, per-group histogram of binned scores
 //                                          (skipped for integer budgets)
 //            select_kernel       Sec. 3.2  threshold bin, its candidates, exact k_hi-th (score, index) key
-//            quant_pack_kernel   Eq. 3-4, Sec. 3.2-3.4  bit map + offsets (prefix over CTAs), pivot test,
+//            quant_pack_stream_kernel (tahq_stream.cuh; tiles owned by one lane, G = 32, 64)
+//            quant_pack_kernel        (tiles owned by two lanes, G = 128)
+//                                Eq. 3-4, Sec. 3.2-3.4  bit map + offsets (prefix over CTAs), pivot test,
 //                                          swap + Hadamard, quantise, pack
 //   decode:  decode_kernel       Sec. 3.3, Alg. 1 l.5  header check, offsets from the bit map, unpack,
 //                                          z + q*s, inverse transform, store
@@ -13,12 +15,6 @@
 
 namespace tahq {
 
-#ifndef TAHQ_STATS_OCC
-#define TAHQ_STATS_OCC 2
-#endif
-#ifndef TAHQ_STATS_NST
-#define TAHQ_STATS_NST 2
-#endif
 
 struct Args {
   const uint8_t *in;        // encode: tensor; decode: unused
@@ -138,7 +134,7 @@ __device__ __forceinline__ uint64_t cta_exclusive_prefix(const Args &a, uint64_t
 // Eq. 1-2: entropy score per tile, plus the per-group histogram of binned scores (Sec. 3.2)
 // ------------------------------------------------------------------------------------------
 template <class C, int NST>
-__global__ void __launch_bounds__(kThreads, TAHQ_STATS_OCC) stats_kernel(const Args a) {
+__global__ void __launch_bounds__(kThreads, 2) stats_kernel(const Args a) {
   extern __shared__ __align__(128) uint8_t smem[];
   __shared__ uint32_t s_hist[kBins];
   const bool use_hist = !a.direct;
@@ -161,11 +157,7 @@ __global__ void __launch_bounds__(kThreads, TAHQ_STATS_OCC) stats_kernel(const A
   long long gcur = -1;
   chunk_pipeline<C, NST>(a.in, a.n_tiles, c0, c1, smem, [&](uint64_t c, const uint8_t *stage) {
     // small groups are ranked on exact scores; large ones are screened first (see select_kernel)
-#if defined(TAHQ_ABLATE) && (TAHQ_ABLATE & 32)
-    const float s = *reinterpret_cast<const float *>(stage + threadIdx.x * 16);
-#else
     const float s = a.direct ? tile_score<C>(stage, a.eps_l1, a.eps_log) : tile_score_screen<C>(stage, a.eps_l1, a.eps_log);
-#endif
     const uint64_t tile0 = c * C::TPC;
     const uint64_t tile = tile0 + threadIdx.x / C::LPT;
     const bool mine = tile < a.n_tiles && (C::LPT == 1 || !(threadIdx.x & 1));
@@ -275,12 +267,6 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const Args a) {
   const float *sc = a.scores + g * ng;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   auto from_smem = [&](uint64_t i, unsigned long long &key) { key = s_keys[i]; return true; };
-#if defined(TAHQ_ABLATE) && (TAHQ_ABLATE & 16)
-  long long sk_t0 = clock64(), sk_prev = sk_t0; long long sk[6] = {0,0,0,0,0,0};
-#define SEL_TICK(i) do { long long n_ = clock64(); sk[i] += n_ - sk_prev; sk_prev = n_; } while (0)
-#else
-#define SEL_TICK(i) do {} while (0)
-#endif
 
   if (a.direct) {   // small group: rank all of its tiles here (one CTA per group)
     for (uint32_t i = threadIdx.x; i < (uint32_t)ng; i += kSelThreads) s_keys[i] = rank_key(sc[i], i);
@@ -325,7 +311,6 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const Args a) {
   }
   __syncthreads();
   const uint32_t B = s_sel[0], r = s_sel[1];
-  SEL_TICK(0);
 
   // ---- B: the scores so far are screening scores s~ (approximate log2), within kScreenErr of the
   // exact ones, so the exact k_hi-th largest score lies within kScreenErr of bin B.  Tiles whose s~
@@ -358,7 +343,6 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const Args a) {
     }
   }
   __syncthreads();
-  SEL_TICK(1);
   if (threadIdx.x == 0 && s_nabove) atomicAdd(&a.nabove[g], s_nabove);
   {
     const uint32_t nl = s_nlist;
@@ -393,16 +377,11 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const Args a) {
     }
   }
 
-  SEL_TICK(2);
   // ---- C: the CTA that finishes the group last ranks the candidates exactly
   __threadfence();
   __syncthreads();
   if (threadIdx.x == 0) s_last = atomicAdd(&a.done[g], 1u) == a.cpg - 1;
   __syncthreads();
-#if defined(TAHQ_ABLATE) && (TAHQ_ABLATE & 16)
-  SEL_TICK(3);
-  if (threadIdx.x == 0) { for (int i = 0; i < 4; ++i) a.flags[256 + blockIdx.x * 8 + i] = (unsigned long long)sk[i]; a.flags[256 + blockIdx.x * 8 + 6] = s_nlist; }
-#endif
   if (!s_last) return;
   __threadfence();
   const uint32_t n = *reinterpret_cast<volatile uint32_t *>(a.ncand + g);
@@ -442,17 +421,6 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const Args a) {
     });
   }
   if (threadIdx.x == 0) a.theta[g] = t;
-#if defined(TAHQ_ABLATE) && (TAHQ_ABLATE & 16)
-  SEL_TICK(4);
-  if (threadIdx.x == 0) { a.flags[256 + blockIdx.x * 8 + 4] = (unsigned long long)sk[4]; a.flags[256 + blockIdx.x * 8 + 5] = n; }
-#endif
-}
-
-// Is tile `tile` one of the k_hi highest-ranked tiles of its group?
-__device__ __forceinline__ bool tile_is_hi(const Args &a, uint64_t tile) {
-  const uint64_t g = tile / a.tiles_per_group;
-  const uint32_t i = (uint32_t)(tile - g * a.tiles_per_group);
-  return rank_key(__ldg(a.scores + tile), i) >= a.theta[g];
 }
 
 // ------------------------------------------------------------------------------------------
@@ -664,48 +632,11 @@ __device__ __forceinline__ void quantise_pairs(float2 (&p)[NPAIR], float mn, flo
   }
 }
 
-// Unflagged bf16 rows never need their elements widened one by one: min/max run on the packed
-// words, and the quantiser's first operation takes the bf16 half as an operand.
-template <class C>
-__device__ __forceinline__ Quantiser encode_raw_bf16_row(const uint8_t *stage, int row, float mn, float mx,
-                                                          uint32_t bits, uint32_t *dst, bool store) {
-  uint32_t w[C::EPT / 2];
-#pragma unroll
-  for (int q = 0; q < C::CPR; ++q) {
-    const uint4 v = *reinterpret_cast<const uint4 *>(stage + (size_t)phys_chunk<C>(row, q) * 16);
-    w[4 * q] = v.x; w[4 * q + 1] = v.y; w[4 * q + 2] = v.z; w[4 * q + 3] = v.w;
-  }
-  const Quantiser q = make_quantiser(mn, mx, bits);
-  const float ymin = (mn - q.z) * q.inv_s, ymax = (mx - q.z) * q.inv_s;
-  const bool safe = ymin >= -0.4999f && ymax < q.qmax + 0.4999f;
-  const float nz = -q.z;   // x + (-z) is x - z
-  const float2 is = f2(q.inv_s), mg = f2(kMagic);
-  if (__all_sync(__activemask(), safe)) {
-    auto t = [&](int k) {
-      float2 d;
-      bf2_add_f32(w[k >> 1], nz, d.x, d.y);
-      d = fma2(d, is, mg);
-      return (k & 1) ? d.y : d.x;
-    };
-    if (store) pack_row<C::EPT>(t, bits, dst);
-  } else {
-    auto t = [&](int k) {
-      float a, b;
-      bf2_add_f32(w[k >> 1], nz, a, b);
-      return fminf(fmaxf(__fmaf_rn((k & 1) ? b : a, q.inv_s, kMagic), kMagic), kMagic + q.qmax);
-    };
-    if (store) pack_row<C::EPT>(t, bits, dst);
-  }
-  return q;
-}
-
 template <class C, int NST>
 __global__ void __launch_bounds__(kThreads, 2) quant_pack_kernel(const Args a) {
   extern __shared__ __align__(128) uint8_t smem[];
-  __shared__ uint8_t s_perm[kThreads];
+  static_assert(C::LPT == 2, "tiles owned by one lane go through quant_pack_stream_kernel");
   __shared__ uint2 s_cnt[kThreads / 32];
-  __shared__ uint16_t s_rowoff[kThreads];
-  __shared__ float2 s_mnmx[kThreads];
   uint32_t *sz32 = reinterpret_cast<uint32_t *>(a.packed + a.off_sz);
   uint8_t *pivot = a.packed + a.off_pivot;
   uint32_t *bitmap = reinterpret_cast<uint32_t *>(a.packed + a.off_bitmap);
@@ -750,71 +681,8 @@ __global__ void __launch_bounds__(kThreads, 2) quant_pack_kernel(const Args a) {
     const bool hi1 = a.mixed && own < nvalid && cur.is_hi_score(a, sc_stage[own], own);
     const uint64_t goff = (uint64_t)(C::G / 8) * ((uint64_t)a.lo * tile0 + hi_run);
 
-    if constexpr (C::LPT == 1) {
-      // ---- phase 1: thread r looks at tile r: range of the row, and a first look at Eq. 3.  The second-
-      // largest magnitude is at least the smaller of |min| and |max| (they sit at different positions,
-      // or every element is equal), so a tile whose largest magnitude does not exceed
-      // tau * (that + varrho) cannot be flagged; only the others ("maybe") need the exact top two.
-      float mn1, mx1;
-      row_minmax<C>(stage, (int)threadIdx.x, mn1, mx1);
-      const float m_big = fmaxf(fabsf(mn1), fabsf(mx1)), m_small = fminf(fabsf(mn1), fabsf(mx1));
-      const bool maybe1 = m_big > a.tau * (m_small + a.eps_ratio);
-      const Regroup rg = regroup((maybe1 ? 2 : 0) | (hi1 ? 1 : 0), s_perm, s_cnt, [&](const Regroup &r) {
-        s_rowoff[threadIdx.x] = (uint16_t)((C::G / 8) * (a.lo * threadIdx.x + r.hi_before));
-        s_mnmx[threadIdx.x] = make_float2(mn1, mx1);
-        if ((threadIdx.x & 31) == 0) bitmap[tile0 / 32 + (threadIdx.x >> 5)] = r.hi_ballot;
-      });
-      hi_run += rg.total_hi;
-      // ---- phase 2: this thread now owns tile `src` of the chunk
-      const int src = rg.src;
-      const bool maybe = rg.cls & 2;
-      const uint32_t b = a.lo + (rg.cls & 1);
-      const uint64_t tile = tile0 + src;
-      const bool live = (uint32_t)src < nvalid;
-      uint32_t *dst = reinterpret_cast<uint32_t *>(a.packed + a.off_payload + goff + s_rowoff[src]);
-      if (C::BF16 && !maybe) {
-        const float2 mm = s_mnmx[src];
-        const Quantiser q = encode_raw_bf16_row<C>(stage, src, mm.x, mm.y, b, dst, live);
-        if (live) { sz32[tile] = q.sz; pivot[tile] = 0; }
-      } else {
-        float a1 = 0.0f, a2 = 0.0f;
-        bool flag = false;
-        if (maybe) {   // Eq. 3 exactly
-          row_top2<C>(stage, src, a1, a2);
-          const float t1 = a2 + a.eps_ratio;
-          const float t2 = a.tau * t1;
-          flag = a1 > t2;
-        }
-        int d = 0;
-        if (flag) {   // Eq. 4: the pivot swap P_d, done in place in shared memory before the row is loaded
-          d = row_first_index_of<C>(stage, src, a1);
-          row_swap_0_d<C, !C::BF16>(const_cast<uint8_t *>(stage), src, d);
-          asm volatile("" ::: "memory");
-        }
-        float2 p[C::EPT / 2];
-        load_row_pairs<C>(stage, src, p);
-        if (flag) {   // Eq. 4: (1/sqrt G) H_G
-          butterfly2<C::EPT / 2>(p);
-#pragma unroll
-          for (int i = 0; i < C::EPT / 2; ++i)   // scalar products: they are added to right after
-            p[i] = f2(p[i].x * hadamard_scale<C>(), p[i].y * hadamard_scale<C>());
-        }
-        float mn = fminf(p[0].x, p[0].y), mx = fmaxf(p[0].x, p[0].y);
-#pragma unroll
-        for (int i = 1; i < C::EPT / 2; ++i) {
-          mn = fminf(mn, fminf(p[i].x, p[i].y));
-          mx = fmaxf(mx, fmaxf(p[i].x, p[i].y));
-        }
-        const Quantiser q = make_quantiser(mn, mx, b);
-        quantise_pairs<C::EPT / 2>(p, mn, mx, q);
-        if (live) {
-          sz32[tile] = q.sz;
-          pivot[tile] = flag ? (uint8_t)(0x80 | d) : (uint8_t)0;
-          pack_row<C::EPT>([&](int k) { return (k & 1) ? p[k >> 1].y : p[k >> 1].x; }, b, dst);
-        }
-      }
-    } else {
-      // ---- 128-wide tiles: two lanes per tile, no regrouping
+    {
+      // ---- two lanes per tile
       const int half = threadIdx.x & 1;
       const uint64_t tile = tile0 + own;
       uint32_t hi_before, total_hi, tiles16;
@@ -1015,11 +883,7 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const Args a) {
       s_chi[ci] = (uint16_t)m;
     }
     bool stop;
-#if defined(TAHQ_ABLATE) && (TAHQ_ABLATE & 4)
-    stop = false; hi_run = 0; __syncthreads();
-#else
     hi_run = cta_exclusive_prefix(a, mine, refuse, stop);   // barriers inside: s_chi is complete
-#endif
     if (blockIdx.x == gridDim.x - 1 && threadIdx.x == 0 && a.mixed && !stop &&
         hi_run + mine != a.n_groups * a.k_hi)
       atomicOr(a.status, 2u /* TAHQ_DEV_BAD_BITMAP */);
@@ -1054,12 +918,6 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const Args a) {
   uint8_t *ostage = smem + S::ROWS;
   // this thread's pieces of the coalesced copy-out: chunk index i*kThreads + tid sits in row i*(kThreads/CPR) + tid/CPR
   const uint8_t *co_src = ostage + (size_t)((int)threadIdx.x ^ swz<C>((int)threadIdx.x / C::CPR)) * 16;
-#if defined(TAHQ_ABLATE) && (TAHQ_ABLATE & 8)
-  long long tk[6] = {0, 0, 0, 0, 0, 0}; long long tprev = clock64();
-#define TAHQ_TICK(i) do { long long now_ = clock64(); tk[i] += now_ - tprev; tprev = now_; } while (0)
-#else
-#define TAHQ_TICK(i) do {} while (0)
-#endif
   if (nch && threadIdx.x == 0) issue(0, hi_run, 0);
   int stage = 0;
   unsigned phases = 0;   // bit s = parity of stage s's mbarrier phase to wait for
@@ -1067,10 +925,8 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const Args a) {
     const uint32_t hi_here = s_chi[ci];
     if (ci + 1 < nch && threadIdx.x == 0)   // the next chunk goes into the other stage (everyone left it last iteration)
       issue(ci + 1, hi_run + hi_here, stage ^ 1);
-    TAHQ_TICK(0);
     if (!mbar_wait(&s_bar[stage], (phases >> stage) & 1u)) atomicOr(a.status, 4u /* TAHQ_DEV_TIMEOUT */);   // chunk ci has landed
     phases ^= 1u << stage;
-    TAHQ_TICK(1);
 
     const uint8_t *st = smem + (size_t)stage * S::STAGE;
     const uint64_t tile0 = t0 + (uint64_t)ci * C::TPC;
@@ -1091,7 +947,6 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const Args a) {
         s_rowoff[threadIdx.x] = (uint16_t)((C::G / 8) * (a.lo * threadIdx.x + r.hi_before));
       });
       // phase 2: this thread now owns tile `src` of the chunk
-      TAHQ_TICK(2);
       const int src = rg.src;
       const bool flag = rg.cls & 2;
       if ((uint32_t)src < nvalid && fits) {
@@ -1099,12 +954,7 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const Args a) {
         const float s = __half2float(__ushort_as_half((unsigned short)(szw & 0xffffu)));
         const float z = __half2float(__ushort_as_half((unsigned short)(szw >> 16)));
         float x[C::EPT];
-#if defined(TAHQ_ABLATE) && (TAHQ_ABLATE & 1)
-#pragma unroll
-        for (int k = 0; k < C::EPT; ++k) x[k] = s + z * k;
-#else
         load_dequant<C::EPT>(pay + s_rowoff[src], a.lo + (rg.cls & 1), s, z, x);
-#endif
         if (flag) {   // (1/sqrt G) H_G^T = the same butterfly
           butterfly<C::EPT>(x);
 #pragma unroll
@@ -1168,15 +1018,9 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const Args a) {
       for (int q = 0; q < C::CPR; ++q)
         *reinterpret_cast<uint4 *>(ostage + (size_t)phys_chunk<C>((int)threadIdx.x, q) * 16) = row_piece<C>(x, q);
     }
-    TAHQ_TICK(3);
     stage ^= 1;
     __syncthreads();   // the chunk is staged; everyone is done with this input stage
-    TAHQ_TICK(4);
-#if defined(TAHQ_ABLATE) && (TAHQ_ABLATE & 2)
-    if (fits && a.lo == 99) {
-#else
     if (fits) {   // the chunk leaves with coalesced 16-byte stores
-#endif
       uint8_t *gout = a.out + tile0 * (uint64_t)(C::G * C::ESZ) + (size_t)threadIdx.x * 16;
       if (nvalid == (uint32_t)C::TPC) {
 #pragma unroll
@@ -1192,12 +1036,7 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const Args a) {
                 *reinterpret_cast<const uint4 *>(co_src + (size_t)i * kThreads * 16);
       }
     }
-    TAHQ_TICK(5);
   }
-#if defined(TAHQ_ABLATE) && (TAHQ_ABLATE & 8)
-  if (threadIdx.x == 0) for (int i = 0; i < 6; ++i) a.cand[blockIdx.x * 8 + i] = (unsigned long long)tk[i];
-  if (threadIdx.x == 0) a.cand[blockIdx.x * 8 + 6] = nch;
-#endif
 }
 
 }  // namespace tahq
