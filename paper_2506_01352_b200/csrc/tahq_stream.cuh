@@ -133,12 +133,12 @@ __device__ __forceinline__ uint32_t encode_plain_words(const uint32_t (&w)[C::RO
 // Eq. 3-4 + Sec. 3.3-3.4 for a queued row (shared memory): exact pivot test, pivot swap, Hadamard,
 // range, codes, bit stream, stores.
 template <class C>
-__device__ __forceinline__ void encode_queued_row(const Args &a, uint8_t *queue, int row, uint32_t bits,
-                                                  uint32_t *dst, uint32_t *sz, uint8_t *pv) {
+__device__ __noinline__ void encode_queued_row(float tau, float eps_ratio, uint8_t *queue, int row, uint32_t bits,
+                                               uint32_t *dst, uint32_t *sz, uint8_t *pv) {
   float a1, a2;
   row_top2<C>(queue, row, a1, a2);
-  const float t1 = a2 + a.eps_ratio;
-  const float t2 = a.tau * t1;
+  const float t1 = a2 + eps_ratio;
+  const float t2 = tau * t1;
   const bool flag = a1 > t2;   // Eq. 3
   int d = 0;
   if (flag) {   // Eq. 4: the pivot swap P_d, done in shared memory before the row is loaded
@@ -262,7 +262,7 @@ __global__ void __launch_bounds__(kThreads, 2) quant_pack_stream_kernel(const Ar
     if ((uint32_t)lane < f_n) {
       const uint64_t tile = tile_cta + (f_tile >> 1);
       const uint64_t off = (uint64_t)(C::G / 8) * ((uint64_t)a.lo * tile + base_hi + f_hib);
-      encode_queued_row<C>(a, fstage, lane, a.lo + (f_tile & 1u), reinterpret_cast<uint32_t *>(payload + off),
+      encode_queued_row<C>(a.tau, a.eps_ratio, fstage, lane, a.lo + (f_tile & 1u), reinterpret_cast<uint32_t *>(payload + off),
                            sz32 + tile, pivot + tile);
     }
     f_n = 0;
