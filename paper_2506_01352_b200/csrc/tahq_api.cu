@@ -242,10 +242,20 @@ static tahq_status decode_t(const Plan &pl, const Args &a, cudaStream_t st) {
   if (!dev_info(&d)) return TAHQ_ERR_CUDA;
   const uint64_t n_chunks = (a.n_tiles + C::TPC - 1) / C::TPC;
   static std::atomic<int> occ_dec[64];
+  (void)pl;
+  if constexpr (C::LPT == 1) {   // one lane per tile: warps stream units of 32 tiles independently
+    const int smem = DecStreamCfg<C>::TOTAL;
+    const int occ = prepare(decode_stream_kernel<C>, smem, d, occ_dec);
+    if (!occ) return TAHQ_ERR_CUDA;
+    const uint64_t n_units = (a.n_tiles + 31) / 32;
+    TAHQ_LAUNCH("decode", st,
+                decode_stream_kernel<C><<<persistent_grid((n_units + kWarps - 1) / kWarps, d, occ), kThreads, smem,
+                                          st>>>(a));
+    return cudaGetLastError() == cudaSuccess ? TAHQ_OK : TAHQ_ERR_CUDA;
+  }
   const int smem = DecSmem<C>::TOTAL;
   const int occ = prepare(decode_kernel<C>, smem, d, occ_dec);
   if (!occ) return TAHQ_ERR_CUDA;
-  (void)pl;
   unsigned grid = persistent_grid(n_chunks, d, occ);
   const uint64_t need = (n_chunks + kChunkCap - 1) / kChunkCap;   // a CTA keeps its chunks' bit map in shared memory
   if (grid < need) grid = (unsigned)need;

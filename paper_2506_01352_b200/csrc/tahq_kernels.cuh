@@ -614,6 +614,63 @@ __device__ __forceinline__ void pack_row(F &&t, uint32_t bits, uint32_t *dst) {
   }
 }
 
+// The same when the width is a per-lane value of at most 4 bits (the lanes of a warp hold tiles of
+// both widths): codes go eight to a group by one multiply-add chain with the lane's 2^W as the
+// multiplier, a group is W whole bytes, and only the last step -- gluing groups into words, a byte
+// permutation -- and the number of stores depend on W.
+template <int N, class F>
+__device__ __forceinline__ void pack_store_narrow(F &&t, uint32_t W, uint32_t *dst) {
+  constexpr int NG = N / 8;
+  constexpr uint32_t K2 = (uint32_t)((0x4B400000ull * group_ones(2, 8)) & 0xffffffffull);
+  constexpr uint32_t K3 = (uint32_t)((0x4B400000ull * group_ones(3, 8)) & 0xffffffffull);
+  constexpr uint32_t K4 = (uint32_t)((0x4B400000ull * group_ones(4, 8)) & 0xffffffffull);
+  const uint32_t M = 1u << W;
+  const uint32_t KW = W == 4 ? K4 : W == 3 ? K3 : K2;
+  uint32_t g[NG];
+#pragma unroll
+  for (int j = 0; j < NG; ++j) {
+    uint32_t acc = __float_as_uint(t(8 * j + 7));
+#pragma unroll
+    for (int i = 6; i >= 0; --i) acc = acc * M + __float_as_uint(t(8 * j + i));
+    g[j] = acc - KW;
+  }
+  if (W == 4) {
+    if constexpr (N == 64) {
+#pragma unroll
+      for (int j = 0; j < NG / 2; ++j) reinterpret_cast<uint2 *>(dst)[j] = make_uint2(g[2 * j], g[2 * j + 1]);
+    } else {
+#pragma unroll
+      for (int j = 0; j < NG; ++j) dst[j] = g[j];
+    }
+  } else if (W == 3) {
+    uint32_t w[3 * NG / 4];
+#pragma unroll
+    for (int j = 0; j < NG / 4; ++j) {
+      w[3 * j] = __byte_perm(g[4 * j], g[4 * j + 1], 0x4210);
+      w[3 * j + 1] = __byte_perm(g[4 * j + 1], g[4 * j + 2], 0x5421);
+      w[3 * j + 2] = __byte_perm(g[4 * j + 2], g[4 * j + 3], 0x6542);
+    }
+    if constexpr (N == 64) {
+#pragma unroll
+      for (int j = 0; j < 3; ++j) reinterpret_cast<uint2 *>(dst)[j] = make_uint2(w[2 * j], w[2 * j + 1]);
+    } else {
+#pragma unroll
+      for (int j = 0; j < 3 * NG / 4; ++j) dst[j] = w[j];
+    }
+  } else {
+    uint32_t w[NG / 2];
+#pragma unroll
+    for (int j = 0; j < NG / 2; ++j) w[j] = __byte_perm(g[2 * j], g[2 * j + 1], 0x5410);
+    if constexpr (N == 64) {
+#pragma unroll
+      for (int j = 0; j < 2; ++j) reinterpret_cast<uint2 *>(dst)[j] = make_uint2(w[2 * j], w[2 * j + 1]);
+    } else {
+#pragma unroll
+      for (int j = 0; j < NG / 2; ++j) dst[j] = w[j];
+    }
+  }
+}
+
 // The same for a row held as adjacent pairs (two elements per instruction).
 template <int NPAIR>
 __device__ __forceinline__ void quantise_pairs(float2 (&p)[NPAIR], float mn, float mx, const Quantiser &q) {

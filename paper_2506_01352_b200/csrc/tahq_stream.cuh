@@ -106,7 +106,7 @@ __device__ __forceinline__ void words_minmax(const uint32_t (&w)[C::ROWB / 4], f
 // Returns the stored {scale, zero}.
 template <class C>
 __device__ __forceinline__ uint32_t encode_plain_words(const uint32_t (&w)[C::ROWB / 4], float mn, float mx,
-                                                       uint32_t bits, uint32_t *dst) {
+                                                       uint32_t bits, bool narrow, uint32_t *dst) {
   const Quantiser q = make_quantiser(mn, mx, bits);
   const float ymin = (mn - q.z) * q.inv_s, ymax = (mx - q.z) * q.inv_s;
   const bool safe = ymin >= -0.4999f && ymax < q.qmax + 0.4999f;
@@ -126,7 +126,8 @@ __device__ __forceinline__ uint32_t encode_plain_words(const uint32_t (&w)[C::RO
       t[i] = f2(fminf(fmaxf(t[i].x, kMagic), kMagic + q.qmax), fminf(fmaxf(t[i].y, kMagic), kMagic + q.qmax));
   }
   auto tk = [&](int k) { return (k & 1) ? t[k >> 1].y : t[k >> 1].x; };
-  pack_row<C::EPT>(tk, bits, dst);
+  if (narrow) pack_store_narrow<C::EPT>(tk, bits, dst);   // every width of this call is at most 4 bits
+  else pack_row<C::EPT>(tk, bits, dst);
   return q.sz;
 }
 
@@ -134,7 +135,7 @@ __device__ __forceinline__ uint32_t encode_plain_words(const uint32_t (&w)[C::RO
 // range, codes, bit stream, stores.
 template <class C>
 __device__ __noinline__ void encode_queued_row(float tau, float eps_ratio, uint8_t *queue, int row, uint32_t bits,
-                                               uint32_t *dst, uint32_t *sz, uint8_t *pv) {
+                                               bool narrow, uint32_t *dst, uint32_t *sz, uint8_t *pv) {
   float a1, a2;
   row_top2<C>(queue, row, a1, a2);
   const float t1 = a2 + eps_ratio;
@@ -164,7 +165,47 @@ __device__ __noinline__ void encode_queued_row(float tau, float eps_ratio, uint8
   quantise_pairs<C::EPT / 2>(p, mn, mx, q);
   *sz = q.sz;
   *pv = flag ? (uint8_t)(0x80 | d) : (uint8_t)0;
-  pack_row<C::EPT>([&](int k) { return (k & 1) ? p[k >> 1].y : p[k >> 1].x; }, bits, dst);
+  auto tk = [&](int k) { return (k & 1) ? p[k >> 1].y : p[k >> 1].x; };
+  if (narrow) pack_store_narrow<C::EPT>(tk, bits, dst);
+  else pack_row<C::EPT>(tk, bits, dst);
+}
+
+// Exclusive running count of set bits over the nw bit-map words of a segment (barriers inside):
+// s_pre[i] = first + bits of words before i; returns the segment's total.
+__device__ __forceinline__ uint32_t scan_segment(const uint32_t *s_bm, uint32_t nw, uint32_t first, uint32_t *s_pre,
+                                                 uint32_t *s_wsum) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  constexpr int PER = kSegWords / kThreads;
+  uint32_t c[PER], mine = 0;
+#pragma unroll
+  for (int j = 0; j < PER; ++j) {
+    const uint32_t i = threadIdx.x * PER + j;
+    c[j] = i < nw ? (uint32_t)__popc(s_bm[i]) : 0u;
+    mine += c[j];
+  }
+  uint32_t incl = mine;
+#pragma unroll
+  for (int o = 1; o < 32; o *= 2) {
+    const uint32_t v = __shfl_up_sync(kFull, incl, o);
+    if (lane >= o) incl += v;
+  }
+  if (lane == 31) s_wsum[warp] = incl;
+  __syncthreads();
+  uint32_t before = incl - mine + first, total = 0;
+#pragma unroll
+  for (int w = 0; w < kWarps; ++w) {
+    const uint32_t v = s_wsum[w];
+    before += w < warp ? v : 0u;
+    total += v;
+  }
+#pragma unroll
+  for (int j = 0; j < PER; ++j) {
+    const uint32_t i = threadIdx.x * PER + j;
+    if (i < nw) s_pre[i] = before;
+    before += c[j];
+  }
+  __syncthreads();
+  return total;
 }
 
 constexpr int kQueueCap = 64;   // tile indices a warp can hold back (32 left over + 32 of one unit)
@@ -239,6 +280,7 @@ __global__ void __launch_bounds__(kThreads, 2) quant_pack_stream_kernel(const Ar
   uint32_t f_n = 0;             // rows on their way into (or waiting in) fstage
   uint32_t f_tile = 0, f_hib = 0;   // lane j's row of fstage
   const uint64_t row_bytes = (uint64_t)C::ROWB;
+  const bool narrow = a.lo + a.mixed <= 4u;   // no width above 4 bits in this call
 
   // fetch the rows of the first n (<= 32) queued tiles again; lane j keeps the j-th tile's particulars
   auto gather = [&](uint32_t n) {
@@ -262,7 +304,8 @@ __global__ void __launch_bounds__(kThreads, 2) quant_pack_stream_kernel(const Ar
     if ((uint32_t)lane < f_n) {
       const uint64_t tile = tile_cta + (f_tile >> 1);
       const uint64_t off = (uint64_t)(C::G / 8) * ((uint64_t)a.lo * tile + base_hi + f_hib);
-      encode_queued_row<C>(a.tau, a.eps_ratio, fstage, lane, a.lo + (f_tile & 1u), reinterpret_cast<uint32_t *>(payload + off),
+      encode_queued_row<C>(a.tau, a.eps_ratio, fstage, lane, a.lo + (f_tile & 1u), narrow,
+                           reinterpret_cast<uint32_t *>(payload + off),
                            sz32 + tile, pivot + tile);
     }
     f_n = 0;
@@ -297,41 +340,7 @@ __global__ void __launch_bounds__(kThreads, 2) quant_pack_stream_kernel(const Ar
       }
     }
     __syncthreads();
-    // ---- exclusive running count of higher-width tiles over the segment's words
-    uint32_t seg_total;
-    {
-      constexpr int PER = kSegWords / kThreads;
-      uint32_t c[PER], mine = 0;
-#pragma unroll
-      for (int j = 0; j < PER; ++j) {
-        const uint32_t i = threadIdx.x * PER + j;
-        c[j] = i < nw ? (uint32_t)__popc(s_bm[i]) : 0u;
-        mine += c[j];
-      }
-      uint32_t incl = mine;
-#pragma unroll
-      for (int o = 1; o < 32; o *= 2) {
-        const uint32_t v = __shfl_up_sync(kFull, incl, o);
-        if (lane >= o) incl += v;
-      }
-      if (lane == 31) s_wsum[warp] = incl;
-      __syncthreads();
-      uint32_t before = incl - mine, total = 0;
-#pragma unroll
-      for (int w = 0; w < kWarps; ++w) {
-        const uint32_t v = s_wsum[w];
-        before += w < warp ? v : 0u;
-        total += v;
-      }
-      seg_total = total;
-      before += seg_hi;
-#pragma unroll
-      for (int j = 0; j < PER; ++j) {
-        const uint32_t i = threadIdx.x * PER + j;
-        if (i < nw) s_pre[i] = before;
-        before += c[j];
-      }
-    }
+    const uint32_t seg_total = scan_segment(s_bm, nw, seg_hi, s_pre, s_wsum);
     if (s0 == u0 && a.mixed) {   // Sec. 3.4: higher-width tiles of all CTAs before this one
       bool unused;
       base_hi = cta_exclusive_prefix(a, single ? (uint64_t)seg_total : counted, false, unused);
@@ -379,7 +388,7 @@ __global__ void __launch_bounds__(kThreads, 2) quant_pack_stream_kernel(const Ar
       qn += (uint32_t)__popc(held);
       if (live && !maybe) {
         const uint64_t off = (uint64_t)(C::G / 8) * ((uint64_t)a.lo * tile + base_hi + hib);
-        sz32[tile] = encode_plain_words<C>(w, mn, mx, a.lo + hi, reinterpret_cast<uint32_t *>(payload + off));
+        sz32[tile] = encode_plain_words<C>(w, mn, mx, a.lo + hi, narrow, reinterpret_cast<uint32_t *>(payload + off));
         pivot[tile] = 0;
       }
       __syncwarp();
@@ -396,6 +405,302 @@ __global__ void __launch_bounds__(kThreads, 2) quant_pack_stream_kernel(const Ar
     __syncwarp();
     run_flagged();
   }
+}
+
+// ------------------------------------------------------------------------------------------
+// Decode, warp-streaming (Sec. 3.3, Algorithm 1 line 5)
+// ------------------------------------------------------------------------------------------
+
+// z + q*s for a row of N codes whose width W (2, 3 or 4 bits) is a per-lane value.  The row's bytes
+// are first regrouped into groups of eight codes (W whole bytes each); a code is then masked where it
+// sits, OR-ed into the mantissa of 2^23 (giving 2^23 + q*2^p exactly), and one subtraction and one
+// fused multiply-add with s*2^-p give the same bits as fma((float)q, s, z).
+template <int N>
+__device__ __forceinline__ void dequant_narrow(const uint32_t (&wv)[N / 8], uint32_t W, float s, float z,
+                                               float (&x)[N]) {
+  constexpr int NG = N / 8;
+  uint32_t g[NG];
+  if (W == 4) {
+#pragma unroll
+    for (int j = 0; j < NG; ++j) g[j] = wv[j];
+  } else if (W == 3) {
+#pragma unroll
+    for (int j = 0; j < NG / 4; ++j) {
+      g[4 * j] = wv[3 * j];
+      g[4 * j + 1] = __funnelshift_r(wv[3 * j], wv[3 * j + 1], 24);
+      g[4 * j + 2] = __funnelshift_r(wv[3 * j + 1], wv[3 * j + 2], 16);
+      g[4 * j + 3] = wv[3 * j + 2] >> 8;
+    }
+  } else {
+#pragma unroll
+    for (int j = 0; j < NG / 2; ++j) {
+      g[2 * j] = wv[j];
+      g[2 * j + 1] = wv[j] >> 16;
+    }
+  }
+  uint32_t two23;
+  asm volatile("mov.u32 %0, 0x4B000000;" : "=r"(two23));
+  const uint32_t M = (1u << W) - 1u, half = 4u * W;
+  uint32_t mk[4];
+  float sc[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    mk[i] = M << (W * i);
+    sc[i] = s * __uint_as_float((127u - W * i) << 23);   // s * 2^-(W i), exact
+  }
+#pragma unroll
+  for (int j = 0; j < NG; ++j) {
+    const uint32_t lo = g[j], hi = g[j] >> half;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      uint32_t m;
+      asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(m) : "r"(i < 4 ? lo : hi), "r"(mk[i & 3]), "r"(two23));
+      const float f = __uint_as_float(m) - 8388608.0f;   // q * 2^p, exact
+      x[8 * j + i] = __fmaf_rn(f, sc[i & 3], z);
+    }
+  }
+}
+
+// The row's codes (shared or global memory, 8-byte aligned for 64-wide rows) -> z + q*s.
+template <class C>
+__device__ __forceinline__ void dequant_row(const uint8_t *src, uint32_t bits, bool narrow, float s, float z,
+                                            float (&x)[C::EPT]) {
+  if (narrow) {
+    uint32_t wv[C::EPT / 8];
+    if constexpr (C::EPT == 64) {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        if (j < 2 || (uint32_t)j < bits) {   // never past the row's own bytes
+          const uint2 v = reinterpret_cast<const uint2 *>(src)[j];
+          wv[2 * j] = v.x; wv[2 * j + 1] = v.y;
+        } else {
+          wv[2 * j] = 0; wv[2 * j + 1] = 0;
+        }
+      }
+    } else {
+#pragma unroll
+      for (int j = 0; j < C::EPT / 8; ++j) wv[j] = (uint32_t)j < bits ? reinterpret_cast<const uint32_t *>(src)[j] : 0u;
+    }
+    dequant_narrow<C::EPT>(wv, bits, s, z, x);
+  } else {
+    load_dequant<C::EPT>(src, bits, s, z, x);
+  }
+}
+
+// Transformed tiles (Eq. 4 inverted): codes from the packed buffer, z + q*s, the butterfly, the
+// scale, the row into the warp's output stage, coordinates 0 and d swapped back there.
+template <class C>
+__device__ __noinline__ void decode_flagged_row(const uint8_t *codes, uint32_t bits, bool narrow, uint32_t szw,
+                                                uint32_t pvb, uint8_t *ostage, int row) {
+  const float s = __half2float(__ushort_as_half((unsigned short)(szw & 0xffffu)));
+  const float z = __half2float(__ushort_as_half((unsigned short)(szw >> 16)));
+  float x[C::EPT];
+  dequant_row<C>(codes, bits, narrow, s, z, x);
+  butterfly<C::EPT>(x);
+#pragma unroll
+  for (int k = 0; k < C::EPT; ++k) x[k] = x[k] * hadamard_scale<C>();
+#pragma unroll
+  for (int q = 0; q < C::CPR; ++q)
+    *reinterpret_cast<uint4 *>(ostage + (size_t)phys_chunk<C>(row, q) * 16) = row_piece<C>(x, q);
+  asm volatile("" ::: "memory");
+  row_swap_0_d<C, !C::BF16>(ostage, row, pvb & (C::G - 1));   // masked: a foreign buffer cannot reach outside the row
+}
+
+template <class C>
+struct DecStreamCfg {
+  static_assert(C::LPT == 1, "one lane per tile");
+  static constexpr int NST = C::BF16 ? 3 : 2;
+  static constexpr int PAY = 32 * C::EPT + 16;          // a unit's codes at 8 bits, from the 16-byte boundary below
+  static constexpr int SLOT = PAY + 32 * 4 + 32;        // + scale/zero words + pivot bytes
+  static constexpr int OUT = 32 * C::ROWB;              // the unit's rows on their way out
+  static constexpr int WARP = NST * SLOT + OUT;
+  static constexpr int TOTAL = kWarps * WARP;
+};
+
+template <class C>
+__global__ void __launch_bounds__(kThreads, 2) decode_stream_kernel(const Args a) {
+  using S = DecStreamCfg<C>;
+  constexpr int NST = S::NST;
+  extern __shared__ __align__(128) uint8_t smem[];
+  __shared__ uint32_t s_bm[kSegWords];
+  __shared__ uint32_t s_pre[kSegWords];
+  __shared__ uint32_t s_wsum[kWarps];
+  __shared__ uint32_t s_bad;
+  __shared__ uint32_t s_q[kWarps][4][kQueueCap];   // held-back tiles: tile - first tile of the CTA, higher-width tiles
+                                                   // before it (and the width bit), scale/zero word, pivot byte
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const unsigned lt = (1u << lane) - 1u;
+  uint8_t *ring = smem + (size_t)warp * S::WARP;
+  uint8_t *ostage = ring + (size_t)NST * S::SLOT;
+  const uint32_t *bitmap = reinterpret_cast<const uint32_t *>(a.packed + a.off_bitmap);
+  const uint8_t *payload = a.packed + a.off_payload;
+
+  const uint64_t n_units = (a.n_tiles + 31) / 32;
+  const uint64_t u0 = n_units * blockIdx.x / gridDim.x, u1 = n_units * (blockIdx.x + 1ull) / gridDim.x;
+  const uint64_t tile_cta = u0 * 32;
+  const bool narrow = a.lo + a.mixed <= 4u;
+
+  // CTA 0 compares the received header with the one these parameters produce; its verdict travels
+  // with the offset prefix, so a refused buffer leaves the output untouched.
+  bool refuse = false;
+  if (blockIdx.x == 0) {
+    if (threadIdx.x == 0) s_bad = 0;
+    __syncthreads();
+    if (threadIdx.x < 32 && reinterpret_cast<const uint32_t *>(a.packed)[threadIdx.x] != a.header[threadIdx.x]) s_bad = 1;
+    __syncthreads();
+    refuse = s_bad != 0;
+    if (refuse && threadIdx.x == 0) atomicOr(a.status, 1u /* TAHQ_DEV_BAD_HEADER */);
+  }
+  // bit-map word i of the tensor, bits beyond the last tile cleared
+  auto bm_word = [&](uint64_t i) -> uint32_t {
+    if (!a.mixed || refuse) return 0u;
+    const uint64_t left = a.n_tiles - i * 32;
+    return __ldg(bitmap + i) & (left >= 32 ? 0xffffffffu : ((1u << (uint32_t)left) - 1u));
+  };
+  if (u0 == u1) {
+    bool stop;
+    cta_exclusive_prefix(a, 0, refuse, stop);
+    return;
+  }
+  const bool single = u1 - u0 <= (uint64_t)kSegWords;
+  uint64_t counted = 0;
+  if (!single) {
+    uint32_t n = 0;
+    for (uint64_t i = u0 + threadIdx.x; i < u1; i += kThreads) n += __popc(bm_word(i));
+    counted = block_sum(n);
+  }
+
+  uint64_t base_hi = 0;
+  uint32_t seg_hi = 0;
+  uint32_t qhead = 0, qn = 0;
+
+  // cp.async of unit u's codes, scale/zero words and pivot bytes into a slot; `hib` = higher-width tiles
+  // of the CTA before the unit.  A unit whose codes would reach past the payload (corrupt bit map) is
+  // not fetched.
+  auto unit_range = [&](uint64_t u, uint32_t hib, uint32_t word, uint64_t &off, uint32_t &len) {
+    const uint64_t t0 = u * 32;
+    const uint64_t left = a.n_tiles - t0;
+    const uint32_t nv = left < 32 ? (uint32_t)left : 32u;
+    off = (uint64_t)(C::G / 8) * ((uint64_t)a.lo * t0 + base_hi + hib);
+    len = (uint32_t)(C::G / 8) * (a.lo * nv + (uint32_t)__popc(word));
+    return off + len <= a.payload_bytes;
+  };
+  auto issue = [&](uint64_t u, uint32_t su, uint8_t *slot) {   // su = u - first unit of the segment
+    uint64_t off;
+    uint32_t len;
+    if (unit_range(u, s_pre[su], s_bm[su], off, len)) {
+      const uint8_t *src = payload + (off & ~15ull);
+      const uint32_t npieces = ((uint32_t)(off & 15ull) + len + 15u) >> 4;
+      for (uint32_t i = lane; i < npieces; i += 32) cp_async16(slot + (size_t)i * 16, src + (size_t)i * 16, 16);
+      if (lane < 8) cp_async16(slot + S::PAY + lane * 16, a.packed + a.off_sz + u * 128 + lane * 16, 16);
+      else if (lane < 10)
+        cp_async16(slot + S::PAY + 128 + (lane - 8) * 16, a.packed + a.off_pivot + u * 32 + (lane - 8) * 16, 16);
+    }
+  };
+  auto prime = [&](uint64_t s0, uint64_t s1) {
+#pragma unroll
+    for (int st = 0; st < NST; ++st) {
+      const uint64_t u = s0 + warp + (uint64_t)st * kWarps;
+      if (u < s1) issue(u, (uint32_t)(u - s0), ring + (size_t)st * S::SLOT);
+      cp_async_commit();
+    }
+  };
+  // the warp's output stage leaves: row r goes to tile `tile_of(r)` if bit r of `rows` is set
+  auto copy_out = [&](unsigned rows, auto &&tile_of) {
+    __syncwarp();
+#pragma unroll
+    for (int i = 0; i < C::CPR; ++i) {
+      const int piece = i * 32 + lane, r = piece / C::CPR, q = piece % C::CPR;
+      const uint64_t t = tile_of(r);
+      if ((rows >> r) & 1u)
+        *reinterpret_cast<uint4 *>(a.out + t * (uint64_t)C::ROWB + (size_t)q * 16) =
+            *reinterpret_cast<const uint4 *>(ostage + (size_t)phys_chunk<C>(r, q) * 16);
+    }
+    __syncwarp();
+  };
+  // the first n (<= 32) held-back tiles, lane j on the j-th
+  auto run_flagged = [&](uint32_t n) {
+    const uint32_t e = (qhead + lane) & (kQueueCap - 1);
+    const uint32_t ft = s_q[warp][0][e], fh = s_q[warp][1][e];
+    if ((uint32_t)lane < n) {
+      const uint64_t tile = tile_cta + ft;
+      const uint64_t off = (uint64_t)(C::G / 8) * ((uint64_t)a.lo * tile + base_hi + (fh >> 1));
+      decode_flagged_row<C>(payload + off, a.lo + (fh & 1u), narrow, s_q[warp][2][e], s_q[warp][3][e], ostage, lane);
+    }
+    copy_out(n >= 32u ? 0xffffffffu : ((1u << n) - 1u), [&](int r) { return tile_cta + __shfl_sync(kFull, ft, r); });
+    qhead = (qhead + n) & (kQueueCap - 1);
+    qn -= n;
+  };
+
+  for (uint64_t s0 = u0; s0 < u1; s0 += kSegWords) {
+    const uint64_t s1 = s0 + kSegWords < u1 ? s0 + kSegWords : u1;
+    const uint32_t nw = (uint32_t)(s1 - s0);
+    if (s0 != u0) __syncthreads();   // every warp is done with the previous segment's words
+    for (uint32_t i = threadIdx.x; i < nw; i += kThreads) s_bm[i] = bm_word(s0 + i);
+    __syncthreads();
+    const uint32_t seg_total = scan_segment(s_bm, nw, seg_hi, s_pre, s_wsum);
+    if (s0 == u0) {   // Sec. 3.4: higher-width tiles of all CTAs before this one; the header's verdict
+      bool stop;
+      const uint64_t mine = single ? (uint64_t)seg_total : counted;
+      base_hi = cta_exclusive_prefix(a, mine, refuse, stop);
+      if (blockIdx.x == gridDim.x - 1 && threadIdx.x == 0 && a.mixed && !stop && base_hi + mine != a.n_groups * a.k_hi)
+        atomicOr(a.status, 2u /* TAHQ_DEV_BAD_BITMAP */);
+      if (stop) return;
+    }
+    prime(s0, s1);
+
+    int slot_i = 0;
+    for (uint64_t u = s0 + warp; u < s1; u += kWarps) {
+      cp_async_wait<NST - 1>();
+      __syncwarp();
+      if (qn >= 32u) run_flagged(32u);
+
+      const uint32_t su = (uint32_t)(u - s0);
+      uint8_t *slot = ring + (size_t)slot_i * S::SLOT;
+      const uint32_t word = s_bm[su];
+      const uint32_t hi = (word >> lane) & 1u;
+      const uint32_t hib = s_pre[su] + (uint32_t)__popc(word & lt);
+      const uint64_t tile = u * 32 + lane;
+      uint64_t off;
+      uint32_t len;
+      const bool fits = unit_range(u, s_pre[su], word, off, len);
+      const bool live = tile < a.n_tiles && fits;
+      const uint32_t szw = reinterpret_cast<const uint32_t *>(slot + S::PAY)[lane];
+      const uint32_t pvb = live ? slot[S::PAY + 128 + lane] : 0u;
+      const bool flagged = (pvb & 0x80u) != 0;
+      const unsigned held = __ballot_sync(kFull, flagged);
+      if (flagged) {   // Eq. 4 inverted costs three times the plain path: held back until 32 have gathered
+        const uint32_t e = (qhead + qn + (uint32_t)__popc(held & lt)) & (kQueueCap - 1);
+        s_q[warp][0][e] = (uint32_t)(tile - tile_cta);
+        s_q[warp][1][e] = (hib << 1) | hi;
+        s_q[warp][2][e] = szw;
+        s_q[warp][3][e] = pvb;
+      }
+      qn += (uint32_t)__popc(held);
+      if (live && !flagged) {
+        const float s = __half2float(__ushort_as_half((unsigned short)(szw & 0xffffu)));
+        const float z = __half2float(__ushort_as_half((unsigned short)(szw >> 16)));
+        const uint8_t *codes = slot + (uint32_t)(off & 15ull) + (uint32_t)(C::G / 8) * (a.lo * lane + (hib - s_pre[su]));
+        float x[C::EPT];
+        dequant_row<C>(codes, a.lo + hi, narrow, s, z, x);
+#pragma unroll
+        for (int q = 0; q < C::CPR; ++q)
+          *reinterpret_cast<uint4 *>(ostage + (size_t)phys_chunk<C>(lane, q) * 16) = row_piece<C>(x, q);
+      }
+      __syncwarp();
+      {   // the slot is free again
+        const uint64_t un = u + (uint64_t)NST * kWarps;
+        if (un < s1) issue(un, (uint32_t)(un - s0), slot);
+        cp_async_commit();
+      }
+      slot_i = (slot_i + 1 == NST) ? 0 : slot_i + 1;
+      copy_out(__ballot_sync(kFull, live && !flagged), [&](int r) { return u * 32 + (uint64_t)r; });
+    }
+    cp_async_wait<0>();
+    __syncwarp();
+    seg_hi += seg_total;
+  }
+  while (qn) run_flagged(qn < 32u ? qn : 32u);
 }
 
 }  // namespace tahq
