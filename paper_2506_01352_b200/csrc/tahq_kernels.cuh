@@ -671,19 +671,21 @@ __device__ __forceinline__ void pack_store_narrow(F &&t, uint32_t W, uint32_t *d
   }
 }
 
-// The same for a row held as adjacent pairs (two elements per instruction).
+// The same for a row held as adjacent pairs (two elements per instruction).  The row's values are
+// pre * p[i] with pre a power of two (an exact product): fma(p, pre, -z) is then the binary32
+// difference (pre * p) - z, and mn, mx are the extremes of the scaled row.
 template <int NPAIR>
-__device__ __forceinline__ void quantise_pairs(float2 (&p)[NPAIR], float mn, float mx, const Quantiser &q) {
+__device__ __forceinline__ void quantise_pairs(float2 (&p)[NPAIR], float pre, float mn, float mx, const Quantiser &q) {
   const float ymin = (mn - q.z) * q.inv_s, ymax = (mx - q.z) * q.inv_s;
   const bool safe = ymin >= -0.4999f && ymax < q.qmax + 0.4999f;
-  const float2 nz = f2(-q.z), is = f2(q.inv_s), mg = f2(kMagic);
+  const float2 nz = f2(-q.z), is = f2(q.inv_s), mg = f2(kMagic), pr = f2(pre);
   if (__all_sync(__activemask(), safe)) {
 #pragma unroll
-    for (int i = 0; i < NPAIR; ++i) p[i] = fma2(add2(p[i], nz), is, mg);
+    for (int i = 0; i < NPAIR; ++i) p[i] = fma2(fma2(p[i], pr, nz), is, mg);
   } else {
 #pragma unroll
     for (int i = 0; i < NPAIR; ++i) {
-      const float2 t = fma2(add2(p[i], nz), is, mg);
+      const float2 t = fma2(fma2(p[i], pr, nz), is, mg);
       p[i] = f2(fminf(fmaxf(t.x, kMagic), kMagic + q.qmax), fminf(fmaxf(t.y, kMagic), kMagic + q.qmax));
     }
   }

@@ -149,11 +149,16 @@ __device__ __noinline__ void encode_queued_row(float tau, float eps_ratio, uint8
   }
   float2 p[C::EPT / 2];
   load_row_pairs<C>(queue, row, p);
-  if (flag) {   // Eq. 4: (1/sqrt G) H_G
+  // Eq. 4: (1/sqrt G) H_G.  For G = 64 the factor is a power of two: the products are exact, so the
+  // factor is applied to the range and inside the quantiser's subtraction instead of element by element.
+  constexpr bool kFold = C::G == 64;
+  if (flag) {
     butterfly2<C::EPT / 2>(p);
+    if (!kFold) {
 #pragma unroll
-    for (int i = 0; i < C::EPT / 2; ++i)   // scalar products: they are added to right after
-      p[i] = f2(p[i].x * hadamard_scale<C>(), p[i].y * hadamard_scale<C>());
+      for (int i = 0; i < C::EPT / 2; ++i)   // scalar products: they are added to right after
+        p[i] = f2(p[i].x * hadamard_scale<C>(), p[i].y * hadamard_scale<C>());
+    }
   }
   float mn = fminf(p[0].x, p[0].y), mx = fmaxf(p[0].x, p[0].y);
 #pragma unroll
@@ -161,8 +166,11 @@ __device__ __noinline__ void encode_queued_row(float tau, float eps_ratio, uint8
     mn = fminf(mn, fminf(p[i].x, p[i].y));
     mx = fmaxf(mx, fmaxf(p[i].x, p[i].y));
   }
+  const float pre = (kFold && flag) ? hadamard_scale<C>() : 1.0f;
+  mn *= pre;
+  mx *= pre;
   const Quantiser q = make_quantiser(mn, mx, bits);
-  quantise_pairs<C::EPT / 2>(p, mn, mx, q);
+  quantise_pairs<C::EPT / 2>(p, pre, mn, mx, q);
   *sz = q.sz;
   *pv = flag ? (uint8_t)(0x80 | d) : (uint8_t)0;
   auto tk = [&](int k) { return (k & 1) ? p[k >> 1].y : p[k >> 1].x; };
@@ -492,13 +500,24 @@ __device__ __forceinline__ void dequant_row(const uint8_t *src, uint32_t bits, b
 template <class C>
 __device__ __noinline__ void decode_flagged_row(const uint8_t *codes, uint32_t bits, bool narrow, uint32_t szw,
                                                 uint32_t pvb, uint8_t *ostage, int row) {
-  const float s = __half2float(__ushort_as_half((unsigned short)(szw & 0xffffu)));
-  const float z = __half2float(__ushort_as_half((unsigned short)(szw >> 16)));
+  float s = __half2float(__ushort_as_half((unsigned short)(szw & 0xffffu)));
+  float z = __half2float(__ushort_as_half((unsigned short)(szw >> 16)));
+  // 1/sqrt(G) is a power of two for G = 64: scaling s and z by it beforehand scales every later value
+  // by it exactly, so the result has the same bits as multiplying at the end
+  constexpr bool kFold = C::G == 64;
+  if (kFold) { s *= hadamard_scale<C>(); z *= hadamard_scale<C>(); }
   float x[C::EPT];
   dequant_row<C>(codes, bits, narrow, s, z, x);
-  butterfly<C::EPT>(x);
+  float2 p[C::EPT / 2];
 #pragma unroll
-  for (int k = 0; k < C::EPT; ++k) x[k] = x[k] * hadamard_scale<C>();
+  for (int i = 0; i < C::EPT / 2; ++i) p[i] = f2(x[2 * i], x[2 * i + 1]);
+  butterfly2<C::EPT / 2>(p);
+  if (!kFold) {
+#pragma unroll
+    for (int i = 0; i < C::EPT / 2; ++i) p[i] = mul2(p[i], f2(hadamard_scale<C>()));   // feeds no addition
+  }
+#pragma unroll
+  for (int i = 0; i < C::EPT / 2; ++i) { x[2 * i] = p[i].x; x[2 * i + 1] = p[i].y; }
 #pragma unroll
   for (int q = 0; q < C::CPR; ++q)
     *reinterpret_cast<uint4 *>(ostage + (size_t)phys_chunk<C>(row, q) * 16) = row_piece<C>(x, q);
