@@ -160,6 +160,8 @@ static void fill_args(const tahq_params *p, const Plan &pl, uint8_t *ws, Args *a
   a->cand_cap = pl.cand_cap;
   a->cpg = pl.cpg;
   a->direct = pl.direct;
+  // the screening score leaves varsigma out; its share of the score is below G * varsigma / ln 2
+  a->exact_scores = pl.direct || (double)p->tile * (double)p->eps_log > 1e-5;
   fill_header(p, pl, a->header);
 }
 
@@ -203,11 +205,22 @@ static tahq_status encode_t(const Plan &pl, const Args &a, cudaStream_t st) {
   const uint64_t n_chunks = (a.n_tiles + C::TPC - 1) / C::TPC;
   static std::atomic<int> occ_stats[64], occ_quant[64], sel_ready[64];
   if (pl.mixed) {
-    constexpr int NS = Stages<C>::STATS;
-    const int smem = NS * C::STAGE_BYTES;
-    const int occ = prepare(stats_kernel<C, NS>, smem, d, occ_stats);
-    if (!occ) return TAHQ_ERR_CUDA;
-    TAHQ_LAUNCH("stats", st, stats_kernel<C, NS><<<persistent_grid(n_chunks, d, occ), kThreads, smem, st>>>(a));
+    if constexpr (C::LPT == 1) {
+      constexpr int NS = C::ROWB <= 128 ? 3 : 2;
+      const int smem = kWarps * NS * StreamCfg<C>::UNIT_BYTES;
+      const int occ = prepare(stats_stream_kernel<C, NS>, smem, d, occ_stats);
+      if (!occ) return TAHQ_ERR_CUDA;
+      const uint64_t n_units = (a.n_tiles + 31) / 32;
+      TAHQ_LAUNCH("stats", st,
+                  stats_stream_kernel<C, NS><<<persistent_grid((n_units + kWarps - 1) / kWarps, d, occ), kThreads, smem,
+                                               st>>>(a));
+    } else {
+      constexpr int NS = Stages<C>::STATS;
+      const int smem = NS * C::STAGE_BYTES;
+      const int occ = prepare(stats_kernel<C, NS>, smem, d, occ_stats);
+      if (!occ) return TAHQ_ERR_CUDA;
+      TAHQ_LAUNCH("stats", st, stats_kernel<C, NS><<<persistent_grid(n_chunks, d, occ), kThreads, smem, st>>>(a));
+    }
     const int sel_smem = kSortCap * 8;
     if (!sel_ready[d.dev & 63].load(std::memory_order_acquire)) {
       if (cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, sel_smem) != cudaSuccess)

@@ -273,8 +273,7 @@ __device__ __forceinline__ void load_abs_oct(const uint8_t *stage, int row, int 
 // Entropy score of the tile this thread (pair) owns: -sum p log2(p + varsigma), p = |a| / (L1 + eps).
 // Two streaming passes over the row in shared memory, eight elements at a time.
 template <class C>
-__device__ __forceinline__ float tile_score(const uint8_t *stage, float eps_l1, float eps_log) {
-  const int row = (int)threadIdx.x;
+__device__ __forceinline__ float tile_score(const uint8_t *stage, int row, float eps_l1, float eps_log) {
   float part[C::NOCT];
 #pragma unroll
   for (int o = 0; o < C::NOCT; ++o) {
@@ -301,41 +300,53 @@ __device__ __forceinline__ float tile_score(const uint8_t *stage, float eps_l1, 
   return 0.0f - S;
 }
 
-// ---- Screening score: the same sums with the hardware's approximate log2 (one MUFU instruction
-// instead of ten FMA-pipe instructions per element).  It is only used to decide which tiles are
-// far enough from a group's threshold to be classified without their exact score; see select_kernel.
+// ---- Screening score: an approximation of the score that costs one pass and one MUFU instruction per
+// element.  With L' = L1 + eps and p = a / L', and leaving varsigma out of the logarithm,
+//     -sum p log2 p  =  ( log2(L') * sum a  -  sum a log2 a ) / L',
+// so the two sums are accumulated together and L' is needed only at the end.  Every magnitude gets
+// 1e-30 added (for free, inside the widening addition) so that a zero contributes 0 * log2(1e-30) = 0.
+// Distance from the exact score: what varsigma contributes, below G * varsigma / ln 2 (the host only
+// selects this function when that is at most 1.5e-5); the hardware log2 (2^-22) and the rounding of
+// the sums, each weighted by p or by |log2 a| <= 127 times a few units in the last place: under 1e-4
+// in all.  It is only used to decide which tiles are far enough from a group's threshold to be
+// classified without their exact score; see select_kernel.
 __device__ __forceinline__ float lg2_approx(float x) {
   float y;
   asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
 template <class C>
-__device__ __forceinline__ float tile_score_screen(const uint8_t *stage, float eps_l1, float eps_log) {
-  const int row = (int)threadIdx.x;
-  float part[C::NOCT];
+__device__ __forceinline__ float tile_score_screen(const uint8_t *stage, int row, float eps_l1) {
+  const float tiny = 1e-30f;
+  float pl[C::NOCT], pt[C::NOCT];
 #pragma unroll
   for (int o = 0; o < C::NOCT; ++o) {
     float v[8];
-    load_abs_oct<C>(stage, row, o, v);
-    part[o] = tree8(v);
-  }
-  float L1 = tree<C::NOCT>(part);
-  if constexpr (C::LPT == 2) L1 = L1 + __shfl_xor_sync(kFull, L1, 1);
-  const float inv = __fdiv_rn(1.0f, L1 + eps_l1);
+    if constexpr (C::BF16) {
+      const uint4 w = *reinterpret_cast<const uint4 *>(stage + (size_t)phys_chunk<C>(row, o) * 16);
+      const uint32_t u[4] = {w.x, w.y, w.z, w.w};
 #pragma unroll
-  for (int o = 0; o < C::NOCT; ++o) {
-    float v[8];
-    load_abs_oct<C>(stage, row, o, v);
+      for (int j = 0; j < 4; ++j) bf2_add_f32(u[j] & 0x7fff7fffu, tiny, v[2 * j], v[2 * j + 1]);
+    } else {
+      load_oct<C>(stage, row, o, v);
 #pragma unroll
-    for (int k = 0; k < 8; ++k) {
-      const float p = v[k] * inv;
-      v[k] = p * lg2_approx(p + eps_log);
+      for (int k = 0; k < 8; ++k) v[k] = fabsf(v[k]) + tiny;
     }
-    part[o] = tree8(v);
+    float t = v[0] * lg2_approx(v[0]);
+#pragma unroll
+    for (int k = 1; k < 8; ++k) t = __fmaf_rn(v[k], lg2_approx(v[k]), t);
+    pt[o] = t;
+    pl[o] = tree8(v);
   }
-  float S = tree<C::NOCT>(part);
-  if constexpr (C::LPT == 2) S = S + __shfl_xor_sync(kFull, S, 1);
-  return 0.0f - S;
+  float L = tree<C::NOCT>(pl), T = tree<C::NOCT>(pt);
+  if constexpr (C::LPT == 2) {
+    L = L + __shfl_xor_sync(kFull, L, 1);
+    T = T + __shfl_xor_sync(kFull, T, 1);
+  }
+  const float Lp = L + eps_l1;
+  float r;
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(Lp));
+  return __fmaf_rn(lg2_approx(Lp), L, -T) * r;
 }
 
 // Exact score of one whole tile read straight from global memory by NOCT neighbouring lanes, lane o

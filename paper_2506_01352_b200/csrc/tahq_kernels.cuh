@@ -34,6 +34,7 @@ struct Args {
   unsigned long long *cand; // [n_groups][cand_cap]
   uint32_t cand_cap, cpg;   // candidate capacity per group; CTAs per group of select_kernel
   uint32_t direct;          // small groups: select_kernel ranks all scores of the group itself
+  uint32_t exact_scores;    // stats_kernel writes exact scores (small groups, or a varsigma too large to screen)
   unsigned long long *flags;// [kMaxGrid] (zeroed per call) per-CTA published counts for the offset prefix
   uint32_t *status;         // device status word
   uint32_t header[32];      // the 128-byte header of the packed buffer
@@ -157,7 +158,8 @@ __global__ void __launch_bounds__(kThreads, 2) stats_kernel(const Args a) {
   long long gcur = -1;
   chunk_pipeline<C, NST>(a.in, a.n_tiles, c0, c1, smem, [&](uint64_t c, const uint8_t *stage) {
     // small groups are ranked on exact scores; large ones are screened first (see select_kernel)
-    const float s = a.direct ? tile_score<C>(stage, a.eps_l1, a.eps_log) : tile_score_screen<C>(stage, a.eps_l1, a.eps_log);
+    const float s = a.exact_scores ? tile_score<C>(stage, (int)threadIdx.x, a.eps_l1, a.eps_log)
+                                   : tile_score_screen<C>(stage, (int)threadIdx.x, a.eps_l1);
     const uint64_t tile0 = c * C::TPC;
     const uint64_t tile = tile0 + threadIdx.x / C::LPT;
     const bool mine = tile < a.n_tiles && (C::LPT == 1 || !(threadIdx.x & 1));

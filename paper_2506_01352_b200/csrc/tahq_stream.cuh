@@ -101,6 +101,73 @@ __device__ __forceinline__ void words_minmax(const uint32_t (&w)[C::ROWB / 4], f
   }
 }
 
+// ------------------------------------------------------------------------------------------
+// Eq. 1-2, warp-streaming: entropy score per tile, per-group histogram of binned scores (Sec. 3.2)
+// ------------------------------------------------------------------------------------------
+template <class C, int NST>
+__global__ void __launch_bounds__(kThreads, 2) stats_stream_kernel(const Args a) {
+  using S = StreamCfg<C>;
+  extern __shared__ __align__(128) uint8_t smem[];
+  __shared__ uint32_t s_hist[kBins];   // this CTA's counts for the ranking group it is in
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  uint8_t *ring = smem + (size_t)warp * NST * S::UNIT_BYTES;
+  const bool use_hist = !a.direct;
+  const uint64_t n_units = (a.n_tiles + 31) / 32;
+  const uint64_t u0 = n_units * blockIdx.x / gridDim.x, u1 = n_units * (blockIdx.x + 1ull) / gridDim.x;
+  if (use_hist)
+    for (int b = threadIdx.x; b < kBins; b += kThreads) s_hist[b] = 0;
+
+  // the CTA's units, one stretch per ranking group: a unit belongs to the group of its first tile
+  uint64_t us = u0;
+  while (us < u1) {
+    const uint64_t g = (us * 32) / a.tiles_per_group;
+    const uint64_t g_end = (g + 1) * a.tiles_per_group;            // first tile of the next group
+    uint64_t ue = (g_end + 31) / 32;
+    if (ue > u1 || !use_hist) ue = u1;
+#pragma unroll
+    for (int s = 0; s < NST; ++s) {
+      const uint64_t u = us + warp + (uint64_t)s * kWarps;
+      if (u < ue) warp_issue_unit<C>(a.in, a.n_tiles, u, ring + (size_t)s * S::UNIT_BYTES, lane);
+      cp_async_commit();
+    }
+    __syncthreads();   // the histogram is clear
+    int slot = 0;
+    for (uint64_t u = us + warp; u < ue; u += kWarps) {
+      cp_async_wait<NST - 1>();
+      __syncwarp();
+      const uint8_t *stage = ring + (size_t)slot * S::UNIT_BYTES;
+      // small groups are ranked on exact scores; large ones are screened first (see select_kernel)
+      const float s = a.exact_scores ? tile_score<C>(stage, lane, a.eps_l1, a.eps_log)
+                                     : tile_score_screen<C>(stage, lane, a.eps_l1);
+      __syncwarp();
+      {
+        const uint64_t un = u + (uint64_t)NST * kWarps;
+        if (un < ue) warp_issue_unit<C>(a.in, a.n_tiles, un, ring + (size_t)slot * S::UNIT_BYTES, lane);
+        cp_async_commit();
+      }
+      slot = (slot + 1 == NST) ? 0 : slot + 1;
+      const uint64_t tile = u * 32 + lane;
+      if (tile < a.n_tiles) {
+        a.scores[tile] = s;
+        if (use_hist) {
+          if (tile < g_end) atomicAdd(&s_hist[score_bin(s)], 1u);
+          else atomicAdd(a.hist + (g + 1) * kBins + score_bin(s), 1u);   // the unit straddles two groups
+        }
+      }
+    }
+    cp_async_wait<0>();
+    __syncthreads();
+    if (use_hist) {   // add this stretch's counts to the group's histogram
+      uint32_t *gh = a.hist + g * kBins;
+      for (int b = threadIdx.x; b < kBins; b += kThreads) {
+        const uint32_t v = s_hist[b];
+        if (v) { atomicAdd(gh + b, v); s_hist[b] = 0; }
+      }
+    }
+    us = ue;
+  }
+}
+
 // Sec. 3.3-3.4 for a row that is not transformed, straight from its raw words: zero-point and scale
 // from the known range, codes (computed once), then the bit stream at the lane's own width.
 // Returns the stored {scale, zero}.

@@ -141,6 +141,37 @@ def test_degenerate_values(kind):
         check_decode(p, packed, want, ws)
 
 
+@pytest.mark.parametrize("scale", [1e-30, 1e-6, 1e-3, 1.0, 300.0, 6e4])
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_selection_survives_input_scale(scale, dtype):
+    """Large ranking groups are selected on approximate scores first; the exact top-k must come out at any
+    magnitude of the input (the entropy score is scale-free, its approximation's rounding is not)."""
+    g = torch.Generator(device="cuda").manual_seed(77)
+    x = torch.randn(320, 2048, generator=g, device="cuda") * torch.exp(torch.randn(320, 1, generator=g, device="cuda"))
+    x[:, ::97] *= 40.0
+    x = (x * scale).to(dtype)
+    p = T.params_for(x, group_tokens=0, tile=64, budget_millibits=3800)      # one group of 10240 tiles
+    packed, want, ws = check_encode(p, x)
+    check_decode(p, packed, want, ws)
+
+
+@pytest.mark.parametrize("eps_log", [1e-8, 1e-4])
+def test_selection_with_near_tied_scores(eps_log):
+    """Many tiles with scores inside one histogram bin of the threshold (rows are permutations and tiny
+    perturbations of one another), and a varsigma too large for the approximate score."""
+    g = torch.Generator(device="cuda").manual_seed(78)
+    base = torch.randn(1, 64, generator=g, device="cuda")
+    rows = []
+    for i in range(10240):
+        perm = torch.randperm(64, generator=g, device="cuda")
+        rows.append(base[0, perm])
+    x = torch.stack(rows).reshape(320, 2048)
+    x = x * (1.0 + 1e-3 * torch.randn(x.shape, generator=g, device="cuda"))
+    p = T.params_for(x, group_tokens=0, tile=64, budget_millibits=3500, eps_log=eps_log)
+    packed, want, ws = check_encode(p, x)
+    check_decode(p, packed, want, ws)
+
+
 def test_decode_refuses_a_foreign_buffer():
     x = synth.make("c1_tiny", device="cuda")
     p = T.params_for(x, group_tokens=64, budget_millibits=3800)
