@@ -264,15 +264,15 @@ static tahq_status decode_t(const Plan &pl, const Args &a, cudaStream_t st) {
     TAHQ_LAUNCH("decode", st,
                 decode_stream_kernel<C><<<persistent_grid((n_units + kWarps - 1) / kWarps, d, occ), kThreads, smem,
                                           st>>>(a));
-    return cudaGetLastError() == cudaSuccess ? TAHQ_OK : TAHQ_ERR_CUDA;
+  } else {
+    const int smem = DecSmem<C>::TOTAL;
+    const int occ = prepare(decode_kernel<C>, smem, d, occ_dec);
+    if (!occ) return TAHQ_ERR_CUDA;
+    unsigned grid = persistent_grid(n_chunks, d, occ);
+    const uint64_t need = (n_chunks + kChunkCap - 1) / kChunkCap;   // a CTA keeps its chunks' bit map in shared memory
+    if (grid < need) grid = (unsigned)need;
+    TAHQ_LAUNCH("decode", st, decode_kernel<C><<<grid, kThreads, smem, st>>>(a));
   }
-  const int smem = DecSmem<C>::TOTAL;
-  const int occ = prepare(decode_kernel<C>, smem, d, occ_dec);
-  if (!occ) return TAHQ_ERR_CUDA;
-  unsigned grid = persistent_grid(n_chunks, d, occ);
-  const uint64_t need = (n_chunks + kChunkCap - 1) / kChunkCap;   // a CTA keeps its chunks' bit map in shared memory
-  if (grid < need) grid = (unsigned)need;
-  TAHQ_LAUNCH("decode", st, decode_kernel<C><<<grid, kThreads, smem, st>>>(a));
   return cudaGetLastError() == cudaSuccess ? TAHQ_OK : TAHQ_ERR_CUDA;
 }
 

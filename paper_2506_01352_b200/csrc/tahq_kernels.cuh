@@ -471,48 +471,6 @@ __device__ __forceinline__ uint32_t block_sum(uint32_t v) {
   return t;
 }
 
-// One-lane-per-tile kernels: stable counting sort of the CTA's 256 tiles by class
-// (bit 0 = higher width, bit 1 = transformed) so that warps become uniform, fused with the running
-// count of higher-width tiles that fixes every tile's payload offset.  `mid` runs between the two
-// barriers (after hi_before / total_hi are known, before the permutation is read).
-struct Regroup {
-  int src, cls;
-  uint32_t hi_before, total_hi, hi_ballot;
-};
-template <class Mid>
-__device__ __forceinline__ Regroup regroup(int cls, uint8_t *s_perm, uint2 *s_cnt, Mid &&mid) {
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const unsigned b1 = __ballot_sync(kFull, cls & 1), b2 = __ballot_sync(kFull, cls & 2);
-  const unsigned m0 = ~b1 & ~b2, m1 = b1 & ~b2, m2 = ~b1 & b2, m3 = b1 & b2;
-  if (lane == 0) s_cnt[warp] = make_uint2(__popc(m0) | (__popc(m1) << 16), __popc(m2) | (__popc(m3) << 16));
-  __syncthreads();
-  uint32_t tot_lo = 0, tot_hi = 0, bef_lo = 0, bef_hi = 0;   // two 16-bit counters per word
-#pragma unroll
-  for (int w = 0; w < kThreads / 32; ++w) {
-    const uint2 c = s_cnt[w];
-    tot_lo += c.x; tot_hi += c.y;
-    bef_lo += (w < warp) ? c.x : 0u;
-    bef_hi += (w < warp) ? c.y : 0u;
-  }
-  const int base1 = tot_lo & 0xffff, base2 = base1 + (tot_lo >> 16), base3 = base2 + (tot_hi & 0xffff);
-  const unsigned mine = (cls == 0) ? m0 : (cls == 1) ? m1 : (cls == 2) ? m2 : m3;
-  const int before = (cls == 0) ? (bef_lo & 0xffff) : (cls == 1) ? (bef_lo >> 16) : (cls == 2) ? (bef_hi & 0xffff)
-                                                                                               : (bef_hi >> 16);
-  const int base = (cls == 0) ? 0 : (cls == 1) ? base1 : (cls == 2) ? base2 : base3;
-  const unsigned lt = (1u << lane) - 1u;
-  Regroup r;
-  r.hi_before = (bef_lo >> 16) + (bef_hi >> 16) + __popc(b1 & lt);
-  r.total_hi = (tot_lo >> 16) + (tot_hi >> 16);
-  r.hi_ballot = b1;
-  mid(r);
-  s_perm[base + before + __popc(mine & lt)] = (uint8_t)threadIdx.x;
-  __syncthreads();
-  r.src = s_perm[threadIdx.x];
-  const int t = threadIdx.x;
-  r.cls = (t >= base1) + (t >= base2) + (t >= base3);
-  return r;
-}
-
 // Two-lanes-per-tile kernels (128-wide tiles): only the running count, no regrouping.
 __device__ __forceinline__ void pair_scan(bool hi, uint32_t *s_cnt32, uint32_t &hi_before, uint32_t &total_hi,
                                           uint32_t &tiles16) {
@@ -895,9 +853,8 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const Args a) {
   constexpr int WPC = C::TPC / 32;          // bit-map words per chunk
   __shared__ uint32_t s_bm[kBmCap];         // bit map of this CTA's tiles (tail bits cleared)
   __shared__ uint16_t s_chi[kChunkCap];     // higher-width tiles per chunk
-  __shared__ uint8_t s_perm[kThreads];
+  static_assert(C::LPT == 2, "tiles owned by one lane go through decode_stream_kernel");
   __shared__ uint2 s_cnt[kThreads / 32];
-  __shared__ uint16_t s_rowoff[kThreads];
   __shared__ uint32_t s_bad;
   const uint32_t *bitmap = reinterpret_cast<const uint32_t *>(a.packed + a.off_bitmap);
   const uint64_t n_chunks = (a.n_tiles + C::TPC - 1) / C::TPC;
@@ -909,7 +866,7 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const Args a) {
     if (threadIdx.x == 0) atomicOr(a.status, 4u);
     return;
   }
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
 
   // CTA 0 compares the received header with the one these parameters produce; its verdict travels
   // with the offset prefix, so a refused buffer leaves the output untouched.
@@ -1000,37 +957,7 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const Args a) {
     const bool fits = goff + (uint64_t)(C::G / 8) * ((uint64_t)a.lo * nvalid + hi_here) <= a.payload_bytes;
     hi_run += hi_here;
 
-    if constexpr (C::LPT == 1) {
-      // phase 1: thread r reads tile r's pivot byte and width bit; the CTA regroups tiles by (transformed?, width)
-      const uint32_t pv1 = threadIdx.x < nvalid ? pv[threadIdx.x] : 0u;
-      const uint32_t hi1 = (s_bm[ci * WPC + warp] >> lane) & 1u;
-      const Regroup rg = regroup(((pv1 & 0x80u) ? 2 : 0) | (int)hi1, s_perm, s_cnt, [&](const Regroup &r) {
-        s_rowoff[threadIdx.x] = (uint16_t)((C::G / 8) * (a.lo * threadIdx.x + r.hi_before));
-      });
-      // phase 2: this thread now owns tile `src` of the chunk
-      const int src = rg.src;
-      const bool flag = rg.cls & 2;
-      if ((uint32_t)src < nvalid && fits) {
-        const uint32_t szw = sz[src];
-        const float s = __half2float(__ushort_as_half((unsigned short)(szw & 0xffffu)));
-        const float z = __half2float(__ushort_as_half((unsigned short)(szw >> 16)));
-        float x[C::EPT];
-        load_dequant<C::EPT>(pay + s_rowoff[src], a.lo + (rg.cls & 1), s, z, x);
-        if (flag) {   // (1/sqrt G) H_G^T = the same butterfly
-          butterfly<C::EPT>(x);
-#pragma unroll
-          for (int k = 0; k < C::EPT; ++k) x[k] = x[k] * hadamard_scale<C>();
-        }
-        uint8_t *orow = ostage + (size_t)src * C::ROWB;
-        const int sx = swz<C>(src) * 16;
-#pragma unroll
-        for (int q = 0; q < C::CPR; ++q) *reinterpret_cast<uint4 *>(orow + ((q * 16) ^ sx)) = row_piece<C>(x, q);
-        if (flag) {   // un-swap coordinates 0 and d in the staged row
-          asm volatile("" ::: "memory");
-          row_swap_0_d<C, !C::BF16>(ostage, src, pv[src] & 0x7f);
-        }
-      }
-    } else {
+    {
       const int half = threadIdx.x & 1;
       const uint32_t own = threadIdx.x >> 1;
       const bool hi1 = (s_bm[ci * WPC + (own >> 5)] >> (own & 31)) & 1u;
