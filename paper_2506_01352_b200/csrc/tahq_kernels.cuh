@@ -584,7 +584,10 @@ __device__ __forceinline__ void pack_store_narrow(F &&t, uint32_t W, uint32_t *d
   constexpr uint32_t K2 = (uint32_t)((0x4B400000ull * group_ones(2, 8)) & 0xffffffffull);
   constexpr uint32_t K3 = (uint32_t)((0x4B400000ull * group_ones(3, 8)) & 0xffffffffull);
   constexpr uint32_t K4 = (uint32_t)((0x4B400000ull * group_ones(4, 8)) & 0xffffffffull);
-  const uint32_t M = 1u << W;
+  // 2^W picked from constants, not shifted: the chain below must stay one multiply-add per code
+  // (a shift and an add would be two instructions, both on the busier ALU pipe)
+  uint32_t M = W == 4 ? 16u : W == 3 ? 8u : 4u;
+  asm volatile("mov.u32 %0, %0;" : "+r"(M));   // opaque to the optimiser: keeps the multiply
   const uint32_t KW = W == 4 ? K4 : W == 3 ? K3 : K2;
   uint32_t g[NG];
 #pragma unroll
