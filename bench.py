@@ -31,16 +31,16 @@ L2_BYTES = 126e6
 # profiles/ (same kernel, same workload); None until a capture exists for that kernel.
 NCU_TRAFFIC_BYTES = {
     # profiles/ncu_full_c3_llama7b_b3800_tile_kernels.md (cold-cache capture, one launch)
-    ("stats", "c3_llama7b", 3800, 64): 68.03e6,
-    ("quant_pack", "c3_llama7b", 3800, 64): 72.53e6,
-    ("decode", "c3_llama7b", 3800, 64): 27.94e6,
+    ("stats", "c3_llama7b", 3800, 64): 67.85e6,
+    ("quant_pack", "c3_llama7b", 3800, 64): 74.73e6,
+    ("decode", "c3_llama7b", 3800, 64): 28.07e6,
 }
 
 
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=40)
+    ap.add_argument("--steps", type=int, default=500)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c3_llama7b")
@@ -77,7 +77,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                 "-lms", "50"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._pump, daemon=True)
             self.thread.start()
         except OSError:
@@ -164,7 +164,7 @@ def main():
     import torch
     import torch.distributed as dist
     from paper_2506_01352_b200 import binding as T
-    from paper_2506_01352_b200 import synth
+    from paper_2506_01352_b200 import shard, synth
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -180,8 +180,8 @@ def main():
     w = synth.WORKLOADS[args.workload]
     n_sets = 4
     # every rank encodes/decodes its own boundary tensors (one per pipeline-stage boundary): no collective
-    xs = [synth.make(args.workload, variant=args.variant, microbatch=rank * n_sets + i, device=dev)
-          for i in range(n_sets)]
+    xs = [synth.make(args.workload, variant=args.variant, microbatch=mb, device=dev)
+          for mb in shard.rank_microbatches(rank, n_sets)]
     p = T.params_for(xs[0], group_tokens=w.seq, tile=args.tile, budget_millibits=args.budget)
     L = T.packed_layout(p)
     in_bytes = xs[0].numel() * xs[0].element_size()
@@ -219,10 +219,7 @@ def main():
             fn(i)
         e1.record(stream)
         barrier()
-        ms = torch.tensor([e0.elapsed_time(e1)], device=dev)
-        if world > 1:
-            dist.all_reduce(ms, op=dist.ReduceOp.MAX)
-        return float(ms.item())
+        return shard.max_over_ranks(e0.elapsed_time(e1), dev)
 
     launches = [0]
 
@@ -284,8 +281,8 @@ def main():
 
     peak, peak_kind = measured_peaks()
     gb = lambda nbytes, ms, steps: nbytes * steps / (ms * 1e-3) / 1e9
-    value = gb(in_bytes * world, ms_total, args.steps)
-    # algorithmic bytes (DESIGN.md section 6): encode reads the tensor once and writes the packed buffer;
+    value = shard.whole_job_rate(in_bytes, world, args.steps, ms_total)
+    # algorithmic bytes: encode reads the tensor once and writes the packed buffer;
     # decode reads the packed buffer and writes the tensor
     alg_dir = in_bytes + packed_bytes
     n_tiles = L["n_tiles"]

@@ -1,0 +1,79 @@
+"""The N > 1 path on CPU: two `gloo` processes.  Ranks take disjoint data, the slowest rank sets the time,
+and a tensor split on ranking-group boundaries encodes to self-contained buffers that decode to the same
+values as the unsplit tensor (the oracle does the arithmetic here; the GPU path is per rank the same call)."""
+import os
+import socket
+
+import numpy as np
+import pytest
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+import oracle as O
+from paper_2506_01352_b200 import shard, synth
+
+
+def _free_port() -> int:
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def _worker(rank: int, world: int, port: int, out):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        # disjoint micro-batches
+        mine = shard.rank_microbatches(rank, 4)
+        got = [None] * world
+        dist.all_gather_object(got, mine)
+        flat = [m for r in got for m in r]
+        assert len(set(flat)) == len(flat) == 4 * world
+
+        # the slowest rank sets the time; the rate counts every rank's bytes
+        ms = shard.max_over_ranks(10.0 + 5.0 * rank)
+        assert ms == 10.0 + 5.0 * (world - 1)
+        assert shard.whole_job_rate(1_000_000, world, 10, ms) == pytest.approx(1e6 * world * 10 / (ms * 1e-3) / 1e9)
+
+        # one tensor split on sample boundaries: every shard's buffer is self-contained
+        x = synth.to_host_array(synth.make("c1_tiny", device="cpu"))          # 128 x 256, groups of 64 tokens
+        tokens, hidden = x.shape
+        first, count = shard.shard_samples(tokens, 64, world, rank)
+        p_all = O.Params(tokens=tokens, hidden=hidden, dtype=0, group_tokens=64, tile=64, budget_millibits=3800)
+        p_me = O.Params(tokens=count, hidden=hidden, dtype=0, group_tokens=64, tile=64, budget_millibits=3800)
+        part = O.decode(p_me, O.encode(p_me, np.ascontiguousarray(x[first:first + count])))
+        whole = O.decode(p_all, O.encode(p_all, x))
+        assert np.array_equal(part, whole[first:first + count])
+        sizes = [None] * world
+        dist.all_gather_object(sizes, (first, count))
+        assert sum(c for _, c in sizes) == tokens and sorted(f for f, _ in sizes)[0] == 0
+        out.put((rank, "ok"))
+    except Exception as e:   # surface the failure in the parent
+        out.put((rank, repr(e)))
+    finally:
+        dist.destroy_process_group()
+
+
+def test_two_ranks_on_gloo():
+    world = 2
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    port = _free_port()
+    procs = [ctx.Process(target=_worker, args=(r, world, port, q)) for r in range(world)]
+    for pr in procs:
+        pr.start()
+    res = dict(q.get(timeout=120) for _ in range(world))
+    for pr in procs:
+        pr.join(timeout=60)
+    assert res == {0: "ok", 1: "ok"}, res
+
+
+@pytest.mark.parametrize("tokens,g,world", [(128, 64, 2), (96, 32, 2), (64, 0, 2), (320, 64, 4), (64, 64, 3)])
+def test_shard_samples_partition(tokens, g, world):
+    spans = [shard.shard_samples(tokens, g, world, r) for r in range(world)]
+    pos = 0
+    for first, count in spans:
+        assert first == pos and count % (g or tokens) == 0
+        pos += count
+    assert pos == tokens
