@@ -37,7 +37,7 @@ typedef struct CUstream_st *tahq_stream;
 typedef enum {
   TAHQ_OK = 0,
   TAHQ_ERR_INVALID_ARG = 1,      /* null pointer, bad struct_size, bad shape/tile/budget        */
-  TAHQ_ERR_UNSUPPORTED = 2,      /* valid in the format but not built (e.g. tile < 32)          */
+  TAHQ_ERR_UNSUPPORTED = 2,      /* valid in the format but not built (tile < 32)               */
   TAHQ_ERR_BUFFER_TOO_SMALL = 3, /* packed_cap / packed_bytes / ws_cap below the bound          */
   TAHQ_ERR_MISALIGNED = 4,       /* a device pointer is not 16-byte aligned                     */
   TAHQ_ERR_CUDA = 5,             /* a CUDA runtime call (launch, memset) failed                 */
@@ -77,8 +77,11 @@ typedef struct {
   float eps_l1;              /* epsilon  of Eq. 1 (1e-8f)                                        */
   float eps_log;             /* varsigma of Eq. 2 (1e-8f); a positive normal binary32 number     */
   float eps_ratio;           /* varrho   of Eq. 3 (1e-8f)                                        */
-  uint32_t rounding;         /* 0 = round-half-even; 1 = stochastic (Philox4x32-10 keyed by seed,
-                                counter = element index / 4)                                     */
+  uint32_t rounding;         /* 0 = round-half-even (the default; the paper names no mode);
+                                1 = stochastic: q = min(floor(clamp(y, 0, 2^b-1) + u), 2^b-1) on the
+                                binary32 product y = (v - z) * (1/s), u = top 24 bits of word (i mod 4)
+                                of Philox4x32-10(key = seed, counter = i / 4) times 2^-24, i = the
+                                element's index in the tensor: codes are a function of (input, seed)  */
   uint64_t seed;             /* used only when rounding == 1                                     */
 } tahq_params;
 

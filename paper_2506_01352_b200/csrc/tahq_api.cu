@@ -80,7 +80,6 @@ static tahq_status make_plan(const tahq_params *p, Plan *pl) {
   L.off_payload = up(L.off_pivot + L.n_tiles, 128);
   L.total_bytes = up(L.off_payload + L.payload_bytes, 128);
   if (G < 32) return TAHQ_ERR_UNSUPPORTED;
-  if (p->rounding != 0) return TAHQ_ERR_UNSUPPORTED;
 
   pl->mixed = L.k_hi > 0;
   pl->direct = L.tiles_per_group <= (uint64_t)kSortCap;
@@ -145,6 +144,7 @@ static void fill_args(const tahq_params *p, const Plan &pl, uint8_t *ws, Args *a
   a->tau = p->tau;
   a->eps_l1 = p->eps_l1;
   a->eps_log = p->eps_log;
+  a->seed = p->seed;
   a->eps_ratio = p->eps_ratio;
   a->status = reinterpret_cast<uint32_t *>(ws);
   a->ncand = reinterpret_cast<uint32_t *>(ws + pl.ws_ncand);
@@ -198,7 +198,7 @@ static unsigned persistent_grid(uint64_t n_chunks, const DevInfo &d, int occ) {
   return (unsigned)(n_chunks < cap ? n_chunks : cap);
 }
 
-template <class C>
+template <class C, bool SR>
 static tahq_status encode_t(const Plan &pl, const Args &a, cudaStream_t st) {
   DevInfo d;
   if (!dev_info(&d)) return TAHQ_ERR_CUDA;
@@ -232,19 +232,19 @@ static tahq_status encode_t(const Plan &pl, const Args &a, cudaStream_t st) {
   if constexpr (C::LPT == 1) {   // one lane per tile: warps stream units of 32 tiles independently
     constexpr int NQ = 2;
     const int smem = StreamCfg<C>::smem_bytes(NQ);
-    const int occ = prepare(quant_pack_stream_kernel<C, NQ>, smem, d, occ_quant);
+    const int occ = prepare(quant_pack_stream_kernel<C, NQ, SR>, smem, d, occ_quant);
     if (!occ) return TAHQ_ERR_CUDA;
     const uint64_t n_units = (a.n_tiles + 31) / 32;
     TAHQ_LAUNCH("quant_pack", st,
-                quant_pack_stream_kernel<C, NQ><<<persistent_grid((n_units + kWarps - 1) / kWarps, d, occ), kThreads,
+                quant_pack_stream_kernel<C, NQ, SR><<<persistent_grid((n_units + kWarps - 1) / kWarps, d, occ), kThreads,
                                                   smem, st>>>(a));
   } else {
     constexpr int NQ = Stages<C>::QUANT;
     const int smem = NQ * (C::STAGE_BYTES + C::TPC * 4);
-    const int occ = prepare(quant_pack_kernel<C, NQ>, smem, d, occ_quant);
+    const int occ = prepare(quant_pack_kernel<C, NQ, SR>, smem, d, occ_quant);
     if (!occ) return TAHQ_ERR_CUDA;
     TAHQ_LAUNCH("quant_pack", st,
-                quant_pack_kernel<C, NQ><<<persistent_grid(n_chunks, d, occ), kThreads, smem, st>>>(a));
+                quant_pack_kernel<C, NQ, SR><<<persistent_grid(n_chunks, d, occ), kThreads, smem, st>>>(a));
   }
   return cudaGetLastError() == cudaSuccess ? TAHQ_OK : TAHQ_ERR_CUDA;
 }
@@ -325,10 +325,17 @@ tahq_status tahq_encode(const tahq_params *p, const void *d_in, void *d_packed, 
   a.packed = static_cast<uint8_t *>(d_packed);
   if (cudaMemsetAsync(d_ws, 0, pl.ws_zero_end, st) != cudaSuccess) return TAHQ_ERR_CUDA;
   const bool bf = p->dtype == TAHQ_BF16;
+  if (p->rounding == 1) {   // stochastic rounding: kernels of their own, the default path carries none of it
+    switch (p->tile) {
+      case 32: return bf ? encode_t<Cfg<32, true>, true>(pl, a, st) : encode_t<Cfg<32, false>, true>(pl, a, st);
+      case 64: return bf ? encode_t<Cfg<64, true>, true>(pl, a, st) : encode_t<Cfg<64, false>, true>(pl, a, st);
+      default: return bf ? encode_t<Cfg<128, true>, true>(pl, a, st) : encode_t<Cfg<128, false>, true>(pl, a, st);
+    }
+  }
   switch (p->tile) {
-    case 32: return bf ? encode_t<Cfg<32, true>>(pl, a, st) : encode_t<Cfg<32, false>>(pl, a, st);
-    case 64: return bf ? encode_t<Cfg<64, true>>(pl, a, st) : encode_t<Cfg<64, false>>(pl, a, st);
-    default: return bf ? encode_t<Cfg<128, true>>(pl, a, st) : encode_t<Cfg<128, false>>(pl, a, st);
+    case 32: return bf ? encode_t<Cfg<32, true>, false>(pl, a, st) : encode_t<Cfg<32, false>, false>(pl, a, st);
+    case 64: return bf ? encode_t<Cfg<64, true>, false>(pl, a, st) : encode_t<Cfg<64, false>, false>(pl, a, st);
+    default: return bf ? encode_t<Cfg<128, true>, false>(pl, a, st) : encode_t<Cfg<128, false>, false>(pl, a, st);
   }
 }
 

@@ -37,6 +37,7 @@ struct Args {
   uint32_t exact_scores;    // stats_kernel writes exact scores (small groups, or a varsigma too large to screen)
   unsigned long long *flags;// [kMaxGrid] (zeroed per call) per-CTA published counts for the offset prefix
   uint32_t *status;         // device status word
+  unsigned long long seed;  // stochastic rounding mode: the generator's key
   uint32_t header[32];      // the 128-byte header of the packed buffer
 };
 
@@ -547,6 +548,45 @@ __device__ __forceinline__ void quantise_row(float (&x)[N], float mn, float mx, 
   }
 }
 
+// Philox4x32 with 10 rounds: the counter-based generator behind the stochastic rounding mode.
+__device__ __forceinline__ void philox4x32_10(uint32_t k0, uint32_t k1, uint32_t c0, uint32_t c1, uint32_t c2,
+                                              uint32_t c3, uint32_t (&out)[4]) {
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    const uint32_t h0 = __umulhi(0xD2511F53u, c0), l0 = 0xD2511F53u * c0;
+    const uint32_t h1 = __umulhi(0xCD9E8D57u, c2), l1 = 0xCD9E8D57u * c2;
+    const uint32_t n0 = h1 ^ c1 ^ k0, n2 = h0 ^ c3 ^ k1;
+    c0 = n0; c1 = l1; c2 = n2; c3 = l0;
+    k0 += 0x9E3779B9u; k1 += 0xBB67AE85u;
+  }
+  out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+// Stochastic rounding mode: d[k] = v_k - z on entry, q_k + 1.5*2^23 on exit, with
+// q_k = min(floor(clamp(d_k * inv_s, 0, qmax) + u_k), qmax) in binary32 and u_k the top 24 bits of
+// word (i mod 4) of Philox(key = seed, counter = i / 4) times 2^-24, i = first + k the element's index
+// in the tensor.  Adding 1.5*2^23 with rounding toward minus infinity is the floor.
+template <int N>
+__device__ __forceinline__ void stochastic_codes(float (&d)[N], float inv_s, float qmax, unsigned long long seed,
+                                                 unsigned long long first) {
+  const uint32_t k0 = (uint32_t)seed, k1 = (uint32_t)(seed >> 32);
+  const unsigned long long c = first >> 2;
+#pragma unroll
+  for (int g = 0; g < N / 4; ++g) {
+    const unsigned long long cg = c + (unsigned)g;
+    uint32_t w[4];
+    philox4x32_10(k0, k1, (uint32_t)cg, (uint32_t)(cg >> 32), 0u, 0u, w);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      float y = __fmul_rn(d[4 * g + j], inv_s);
+      y = fminf(fmaxf(y, 0.0f), qmax);
+      const float u = __fmul_rn(__uint2float_rn(w[j] >> 8), 0x1p-24f);
+      const float t = __fadd_rd(__fadd_rn(y, u), kMagic);
+      d[4 * g + j] = fminf(t, kMagic + qmax);
+    }
+  }
+}
+
 // t(k) must return q_k + 1.5*2^23 for a compile-time k; the row's N*bits/32 words go straight to
 // the payload (rows of 64 codes start on 8-byte boundaries).
 template <int W, int N, class F>
@@ -654,7 +694,7 @@ __device__ __forceinline__ void quantise_pairs(float2 (&p)[NPAIR], float pre, fl
   }
 }
 
-template <class C, int NST>
+template <class C, int NST, bool SR>
 __global__ void __launch_bounds__(kThreads, 2) quant_pack_kernel(const Args a) {
   extern __shared__ __align__(128) uint8_t smem[];
   static_assert(C::LPT == 2, "tiles owned by one lane go through quant_pack_stream_kernel");
@@ -770,7 +810,13 @@ __global__ void __launch_bounds__(kThreads, 2) quant_pack_kernel(const Args a) {
       mn = fminf(mn, __shfl_xor_sync(kFull, mn, 1));
       mx = fmaxf(mx, __shfl_xor_sync(kFull, mx, 1));
       const Quantiser q = make_quantiser(mn, mx, b);
-      quantise_row<C::EPT>(x, mn, mx, q);
+      if constexpr (SR) {
+#pragma unroll
+        for (int k = 0; k < C::EPT; ++k) x[k] = x[k] - q.z;
+        stochastic_codes<C::EPT>(x, q.inv_s, q.qmax, a.seed, tile * (unsigned long long)C::G + (unsigned)(half * C::EPT));
+      } else {
+        quantise_row<C::EPT>(x, mn, mx, q);
+      }
       if (own < nvalid) {
         if (half == 0) {
           sz32[tile] = q.sz;

@@ -171,10 +171,24 @@ __global__ void __launch_bounds__(kThreads, 2) stats_stream_kernel(const Args a)
 // Sec. 3.3-3.4 for a row that is not transformed, straight from its raw words: zero-point and scale
 // from the known range, codes (computed once), then the bit stream at the lane's own width.
 // Returns the stored {scale, zero}.
-template <class C>
+template <class C, bool SR>
 __device__ __forceinline__ uint32_t encode_plain_words(const uint32_t (&w)[C::ROWB / 4], float mn, float mx,
-                                                       uint32_t bits, bool narrow, uint32_t *dst) {
+                                                       uint32_t bits, bool narrow, uint32_t *dst,
+                                                       unsigned long long seed, unsigned long long first) {
   const Quantiser q = make_quantiser(mn, mx, bits);
+  if constexpr (SR) {
+    float d[C::EPT];
+#pragma unroll
+    for (int i = 0; i < C::EPT / 2; ++i) {
+      if constexpr (C::BF16) bf2_add_f32(w[i], -q.z, d[2 * i], d[2 * i + 1]);
+      else { d[2 * i] = __uint_as_float(w[2 * i]) - q.z; d[2 * i + 1] = __uint_as_float(w[2 * i + 1]) - q.z; }
+    }
+    stochastic_codes<C::EPT>(d, q.inv_s, q.qmax, seed, first);
+    auto tk = [&](int k) { return d[k]; };
+    if (narrow) pack_store_narrow<C::EPT>(tk, bits, dst);
+    else pack_row<C::EPT>(tk, bits, dst);
+    return q.sz;
+  }
   const float ymin = (mn - q.z) * q.inv_s, ymax = (mx - q.z) * q.inv_s;
   const bool safe = ymin >= -0.4999f && ymax < q.qmax + 0.4999f;
   const float nz = -q.z;   // x + (-z) is x - z
@@ -200,9 +214,10 @@ __device__ __forceinline__ uint32_t encode_plain_words(const uint32_t (&w)[C::RO
 
 // Eq. 3-4 + Sec. 3.3-3.4 for a queued row (shared memory): exact pivot test, pivot swap, Hadamard,
 // range, codes, bit stream, stores.
-template <class C>
+template <class C, bool SR>
 __device__ __noinline__ void encode_queued_row(float tau, float eps_ratio, uint8_t *queue, int row, uint32_t bits,
-                                               bool narrow, uint32_t *dst, uint32_t *sz, uint8_t *pv) {
+                                               bool narrow, uint32_t *dst, uint32_t *sz, uint8_t *pv,
+                                               unsigned long long seed, unsigned long long first) {
   float a1, a2;
   row_top2<C>(queue, row, a1, a2);
   const float t1 = a2 + eps_ratio;
@@ -237,7 +252,19 @@ __device__ __noinline__ void encode_queued_row(float tau, float eps_ratio, uint8
   mn *= pre;
   mx *= pre;
   const Quantiser q = make_quantiser(mn, mx, bits);
-  quantise_pairs<C::EPT / 2>(p, pre, mn, mx, q);
+  if constexpr (SR) {
+    float d[C::EPT];
+#pragma unroll
+    for (int i = 0; i < C::EPT / 2; ++i) {
+      d[2 * i] = __fmaf_rn(p[i].x, pre, -q.z);
+      d[2 * i + 1] = __fmaf_rn(p[i].y, pre, -q.z);
+    }
+    stochastic_codes<C::EPT>(d, q.inv_s, q.qmax, seed, first);
+#pragma unroll
+    for (int i = 0; i < C::EPT / 2; ++i) p[i] = f2(d[2 * i], d[2 * i + 1]);
+  } else {
+    quantise_pairs<C::EPT / 2>(p, pre, mn, mx, q);
+  }
   *sz = q.sz;
   *pv = flag ? (uint8_t)(0x80 | d) : (uint8_t)0;
   auto tk = [&](int k) { return (k & 1) ? p[k >> 1].y : p[k >> 1].x; };
@@ -285,7 +312,7 @@ __device__ __forceinline__ uint32_t scan_segment(const uint32_t *s_bm, uint32_t 
 
 constexpr int kQueueCap = 64;   // tile indices a warp can hold back (32 left over + 32 of one unit)
 
-template <class C, int NST>
+template <class C, int NST, bool SR>
 __global__ void __launch_bounds__(kThreads, 2) quant_pack_stream_kernel(const Args a) {
   using S = StreamCfg<C>;
   extern __shared__ __align__(128) uint8_t smem[];
@@ -379,9 +406,9 @@ __global__ void __launch_bounds__(kThreads, 2) quant_pack_stream_kernel(const Ar
     if ((uint32_t)lane < f_n) {
       const uint64_t tile = tile_cta + (f_tile >> 1);
       const uint64_t off = (uint64_t)(C::G / 8) * ((uint64_t)a.lo * tile + base_hi + f_hib);
-      encode_queued_row<C>(a.tau, a.eps_ratio, fstage, lane, a.lo + (f_tile & 1u), narrow,
-                           reinterpret_cast<uint32_t *>(payload + off),
-                           sz32 + tile, pivot + tile);
+      encode_queued_row<C, SR>(a.tau, a.eps_ratio, fstage, lane, a.lo + (f_tile & 1u), narrow,
+                               reinterpret_cast<uint32_t *>(payload + off), sz32 + tile, pivot + tile, a.seed,
+                               tile * (unsigned long long)C::G);
     }
     f_n = 0;
     __syncwarp();
@@ -463,7 +490,8 @@ __global__ void __launch_bounds__(kThreads, 2) quant_pack_stream_kernel(const Ar
       qn += (uint32_t)__popc(held);
       if (live && !maybe) {
         const uint64_t off = (uint64_t)(C::G / 8) * ((uint64_t)a.lo * tile + base_hi + hib);
-        sz32[tile] = encode_plain_words<C>(w, mn, mx, a.lo + hi, narrow, reinterpret_cast<uint32_t *>(payload + off));
+        sz32[tile] = encode_plain_words<C, SR>(w, mn, mx, a.lo + hi, narrow, reinterpret_cast<uint32_t *>(payload + off),
+                                               a.seed, tile * (unsigned long long)C::G);
         pivot[tile] = 0;
       }
       __syncwarp();

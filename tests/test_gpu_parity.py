@@ -172,6 +172,33 @@ def test_selection_with_near_tied_scores(eps_log):
     check_decode(p, packed, want, ws)
 
 
+@pytest.mark.parametrize("G", [32, 64, 128])
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_stochastic_rounding_mode(G, dtype):
+    """rounding = 1 (not in the paper): floor(y + u) with u from Philox4x32-10 keyed by the seed and indexed by
+    the element's position in the tensor, so the codes are a pure function of (input, seed) on any machine."""
+    x = synth.make("c1_tiny", device="cuda", microbatch=3).to(dtype)
+    for seed, beta in ((1, 3800), (0xDEADBEEFCAFE, 3000), (7, 6500)):
+        p = T.params_for(x, group_tokens=64, tile=G, budget_millibits=beta, rounding=1, seed=seed)
+        packed, want, ws = check_encode(p, x)
+        check_decode(p, packed, want, ws)
+
+
+def test_stochastic_rounding_large_and_seed_dependent():
+    x = synth.make("c2_gpt2s", device="cuda")
+    p1 = T.params_for(x, group_tokens=1024, tile=64, budget_millibits=3800, rounding=1, seed=11)
+    packed1, want1, ws = check_encode(p1, x)
+    check_decode(p1, packed1, want1, ws)
+    p2 = T.params_for(x, group_tokens=1024, tile=64, budget_millibits=3800, rounding=1, seed=12)
+    packed2 = T.alloc_packed(p2, x.device)
+    T.encode(p2, x, packed=packed2, ws=ws)
+    torch.cuda.synchronize()
+    L = T.packed_layout(p2)
+    a, b = packed1.cpu().numpy(), packed2.cpu().numpy()
+    assert np.array_equal(a[L["off_bitmap"]:L["off_payload"]], b[L["off_bitmap"]:L["off_payload"]])   # same widths, ranges
+    assert not np.array_equal(a[L["off_payload"]:], b[L["off_payload"]:])                             # other draws
+
+
 def test_decode_refuses_a_foreign_buffer():
     x = synth.make("c1_tiny", device="cuda")
     p = T.params_for(x, group_tokens=64, budget_millibits=3800)
