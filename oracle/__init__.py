@@ -16,6 +16,8 @@ import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "tahq_oracle.c")
+_SRC_Q = os.path.join(_HERE, "qnaive_oracle.c")
+_HDR_Q = os.path.join(_HERE, "qnaive_oracle.h")
 _HDR = os.path.join(_HERE, "tahq_oracle.h")
 _LIB = os.path.join(_HERE, "libtahq_oracle.so")
 
@@ -56,6 +58,31 @@ class _Layout(C.Structure):
     ]
 
 
+class _QParams(C.Structure):
+    _fields_ = [("dtype", C.c_uint32), ("tokens", C.c_uint64), ("hidden", C.c_uint32), ("bits", C.c_uint32),
+                ("per_tensor", C.c_uint32), ("prescale", C.c_float)]
+
+
+class _QLayout(C.Structure):
+    _fields_ = [("n_scales", C.c_uint64), ("off_scales", C.c_uint64), ("off_payload", C.c_uint64),
+                ("row_bytes", C.c_uint64), ("total_bytes", C.c_uint64)]
+
+
+@dataclass
+class QNaiveParams:
+    """Fixed-point gradient compressor of Algorithm 1 line 6 (b bits, per-token or per-tensor scale, pre-scale c)."""
+
+    tokens: int
+    hidden: int
+    dtype: int = F32
+    bits: int = 8
+    per_tensor: int = 0
+    prescale: float = 1.0
+
+    def c(self) -> _QParams:
+        return _QParams(self.dtype, self.tokens, self.hidden, self.bits, self.per_tensor, self.prescale)
+
+
 @dataclass
 class Params:
     """Configuration of one boundary tensor (names follow the paper: G, S, tau, ...)."""
@@ -81,11 +108,11 @@ class Params:
 
 def build(force: bool = False) -> str:
     """Compile the oracle with gcc (no contraction, no fast-math); returns the library path."""
-    newest = max(os.path.getmtime(_SRC), os.path.getmtime(_HDR))
+    newest = max(os.path.getmtime(f) for f in (_SRC, _HDR, _SRC_Q, _HDR_Q))
     if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < newest:
         tmp = _LIB + f".tmp{os.getpid()}"
         cmd = ["gcc", "-O2", "-std=c11", "-ffp-contract=off", "-fno-fast-math", "-fopenmp",
-               "-fPIC", "-shared", "-Wall", "-o", tmp, _SRC, "-lm"]
+               "-fPIC", "-shared", "-Wall", "-o", tmp, _SRC, _SRC_Q, "-lm"]
         subprocess.run(cmd, check=True, cwd=_HERE)
         os.replace(tmp, _LIB)
     return _LIB
@@ -127,6 +154,14 @@ def lib() -> C.CDLL:
         L.tahqo_quantise.argtypes = [fp, C.c_uint32, C.c_uint32, C.c_uint16, C.c_uint16,
                                      C.c_uint32, C.c_uint64, C.c_uint64, C.POINTER(C.c_uint32)]
         L.tahqo_philox4x32_10.argtypes = [C.POINTER(C.c_uint32)] * 3
+        L.qnaiveo_layout_of.argtypes = [C.POINTER(_QParams), C.POINTER(_QLayout)]
+        L.qnaiveo_layout_of.restype = C.c_int
+        L.qnaiveo_packed_bound.argtypes = [C.POINTER(_QParams)]
+        L.qnaiveo_packed_bound.restype = C.c_size_t
+        L.qnaiveo_encode.argtypes = [C.POINTER(_QParams), C.c_void_p, C.c_void_p, C.c_size_t]
+        L.qnaiveo_encode.restype = C.c_int
+        L.qnaiveo_decode.argtypes = [C.POINTER(_QParams), C.c_void_p, C.c_size_t, C.c_void_p]
+        L.qnaiveo_decode.restype = C.c_int
         _lib = L
     return _lib
 
@@ -267,3 +302,39 @@ def philox4x32_10(key, ctr) -> np.ndarray:
     o = (C.c_uint32 * 4)()
     lib().tahqo_philox4x32_10(k, c, o)
     return np.array(list(o), dtype=np.uint32)
+
+
+# ---------------------------------------------------------------- fixed-point gradient compressor
+def qnaive_layout(p: QNaiveParams) -> dict:
+    L = _QLayout()
+    if lib().qnaiveo_layout_of(C.byref(p.c()), C.byref(L)):
+        raise ValueError("invalid parameters")
+    return {f: getattr(L, f) for f, _ in _QLayout._fields_}
+
+
+def qnaive_packed_bound(p: QNaiveParams) -> int:
+    return int(lib().qnaiveo_packed_bound(C.byref(p.c())))
+
+
+def qnaive_encode(p: QNaiveParams, x: np.ndarray) -> np.ndarray:
+    want = np.uint16 if p.dtype == BF16 else np.float32
+    x = np.ascontiguousarray(x)
+    if x.dtype != want or x.size != p.tokens * p.hidden:
+        raise ValueError("input does not match the parameters")
+    n = qnaive_packed_bound(p)
+    if n == 0:
+        raise ValueError("invalid parameters")
+    out = np.empty(n, dtype=np.uint8)
+    rc = lib().qnaiveo_encode(C.byref(p.c()), x.ctypes.data, out.ctypes.data, n)
+    if rc:
+        raise RuntimeError(f"qnaiveo_encode failed: {rc}")
+    return out
+
+
+def qnaive_decode(p: QNaiveParams, packed: np.ndarray) -> np.ndarray:
+    packed = np.ascontiguousarray(packed, dtype=np.uint8)
+    out = np.empty((p.tokens, p.hidden), dtype=np.uint16 if p.dtype == BF16 else np.float32)
+    rc = lib().qnaiveo_decode(C.byref(p.c()), packed.ctypes.data, packed.size, out.ctypes.data)
+    if rc:
+        raise RuntimeError(f"qnaiveo_decode failed: {rc}")
+    return out

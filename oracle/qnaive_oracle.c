@@ -1,0 +1,138 @@
+/*
+ * Fixed-point ("naive") gradient compressor -- CPU ORACLE (test infrastructure, not the product).
+ * See qnaive_oracle.h.  Plain scalar C, one loop per step.
+ *
+ * Reading of Q_Naive (the paper names it, Sec. 3.5 and Algorithm 1 line 6, but prints no formula):
+ *   y   = c * g                      binary32 product (appendix: g_hat = Q(c g) / c)
+ *   m   = max |y|                    over one token (row), or over the whole tensor
+ *   L   = 2^(b-1) - 1                symmetric fixed point, b bits, no negative extreme
+ *   s   = m / L                      binary32 division; stored as binary32
+ *   q   = clamp(round(y / s), -L, L) evaluated as y * (1/s) with the product taken exactly and
+ *                                    rounded once, ties to even (1/s = 0 when s = 0)
+ *   code = q + L                     unsigned, b bits, little-endian bit stream per row
+ *   g_hat = (q * s) / c              binary32 product, then binary32 division
+ *
+ * Packed format (little-endian; sections start on 128-byte boundaries; padding is zero):
+ *   header 128 B: "TAHN", version 1, dtype, bits, tokens(u64), hidden, per_tensor, c (f32 bits),
+ *                 row_bytes(u64), total_bytes(u64)
+ *   scales: binary32 per token (or one)
+ *   payload: row r at r * row_bytes, row_bytes = ceil(hidden*b/8) rounded up to 16; element k of a
+ *            row occupies stream bits [k*b, (k+1)*b), stream bit j = byte j>>3 bit j&7.
+ *
+ * Parity unpinned: the paper prints neither a formula nor a worked example for Q_Naive; the pins of
+ * tests/test_oracle_qnaive.py are the textbook expression, the error bound, and the invariances.
+ *
+ * Build: gcc -O2 -std=c11 -ffp-contract=off -fno-fast-math -fPIC -shared
+ */
+#include "qnaive_oracle.h"
+
+#include <math.h>
+#include <string.h>
+
+static uint64_t up(uint64_t x, uint64_t a) { return (x + a - 1) / a * a; }
+static void put32(uint8_t *d, uint32_t v) { for (int i = 0; i < 4; i++) d[i] = (uint8_t)(v >> (8 * i)); }
+static void put64(uint8_t *d, uint64_t v) { for (int i = 0; i < 8; i++) d[i] = (uint8_t)(v >> (8 * i)); }
+static float bf16_to_f32(uint16_t h) { uint32_t u = (uint32_t)h << 16; float x; memcpy(&x, &u, 4); return x; }
+static uint16_t f32_to_bf16(float x) {   /* round to nearest even */
+  uint32_t u; memcpy(&u, &x, 4);
+  if ((u & 0x7fffffffu) > 0x7f800000u) return (uint16_t)((u >> 16) | 0x40u);
+  u += 0x7fffu + ((u >> 16) & 1u);
+  return (uint16_t)(u >> 16);
+}
+
+int qnaiveo_layout_of(const qnaiveo_params *p, qnaiveo_layout *L) {
+  if (!p || !L) return 1;
+  if (p->dtype > 1 || p->per_tensor > 1) return 1;
+  if (p->tokens == 0 || p->hidden == 0 || p->hidden % 8) return 1;
+  if (p->bits < 2 || p->bits > 16) return 1;
+  if (!(p->prescale > 0.0f) || isinf(p->prescale)) return 1;
+  L->n_scales = p->per_tensor ? 1 : p->tokens;
+  L->row_bytes = up(((uint64_t)p->hidden * p->bits + 7) / 8, 16);
+  L->off_scales = 128;
+  L->off_payload = up(L->off_scales + 4 * L->n_scales, 128);
+  L->total_bytes = up(L->off_payload + p->tokens * L->row_bytes, 128);
+  return 0;
+}
+
+size_t qnaiveo_packed_bound(const qnaiveo_params *p) {
+  qnaiveo_layout L;
+  return qnaiveo_layout_of(p, &L) ? 0 : (size_t)L.total_bytes;
+}
+
+static float load(const qnaiveo_params *p, const void *in, uint64_t i) {
+  return p->dtype ? bf16_to_f32(((const uint16_t *)in)[i]) : ((const float *)in)[i];
+}
+
+int qnaiveo_encode(const qnaiveo_params *p, const void *in, uint8_t *packed, size_t cap) {
+  qnaiveo_layout L;
+  if (qnaiveo_layout_of(p, &L) || !in || !packed) return 1;
+  if (cap < L.total_bytes) return 3;
+  memset(packed, 0, (size_t)L.total_bytes);
+  memcpy(packed, "TAHN", 4);
+  put32(packed + 4, 1u);
+  put32(packed + 8, p->dtype);
+  put32(packed + 12, p->bits);
+  put64(packed + 16, p->tokens);
+  put32(packed + 24, p->hidden);
+  put32(packed + 28, p->per_tensor);
+  { uint32_t u; memcpy(&u, &p->prescale, 4); put32(packed + 32, u); }
+  put64(packed + 40, L.row_bytes);
+  put64(packed + 48, L.total_bytes);
+
+  const float c = p->prescale;
+  const float Lq = (float)((1u << (p->bits - 1)) - 1u);
+  const uint64_t C = p->hidden;
+  float m_all = 0.0f;
+  if (p->per_tensor)
+    for (uint64_t i = 0; i < p->tokens * C; i++) m_all = fmaxf(m_all, fabsf(c * load(p, in, i)));
+  for (uint64_t r = 0; r < p->tokens; r++) {
+    float m = m_all;
+    if (!p->per_tensor) {
+      m = 0.0f;
+      for (uint64_t k = 0; k < C; k++) m = fmaxf(m, fabsf(c * load(p, in, r * C + k)));
+    }
+    const float s = m / Lq;
+    const float inv = s > 0.0f ? 1.0f / s : 0.0f;
+    if (!p->per_tensor || r == 0) {
+      uint32_t u; memcpy(&u, &s, 4);
+      put32(packed + L.off_scales + 4 * (p->per_tensor ? 0 : r), u);
+    }
+    uint8_t *row = packed + L.off_payload + r * L.row_bytes;
+    for (uint64_t k = 0; k < C; k++) {
+      const float y = c * load(p, in, r * C + k);
+      double t = (double)y * (double)inv;          /* exact */
+      if (t > (double)Lq) t = (double)Lq;
+      if (t < -(double)Lq) t = -(double)Lq;
+      const int q = (int)rint(t);                  /* nearest, ties to even */
+      const uint32_t code = (uint32_t)(q + (int)Lq);
+      uint64_t bit = k * p->bits;
+      for (uint32_t j = 0; j < p->bits; j++, bit++)
+        if ((code >> j) & 1u) row[bit >> 3] |= (uint8_t)(1u << (bit & 7));
+    }
+  }
+  return 0;
+}
+
+int qnaiveo_decode(const qnaiveo_params *p, const uint8_t *packed, size_t bytes, void *out) {
+  qnaiveo_layout L;
+  if (qnaiveo_layout_of(p, &L) || !packed || !out) return 1;
+  if (bytes < L.total_bytes) return 3;
+  const float c = p->prescale;
+  const int Lq = (int)((1u << (p->bits - 1)) - 1u);
+  const uint64_t C = p->hidden;
+  for (uint64_t r = 0; r < p->tokens; r++) {
+    float s;
+    memcpy(&s, packed + L.off_scales + 4 * (p->per_tensor ? 0 : r), 4);
+    const uint8_t *row = packed + L.off_payload + r * L.row_bytes;
+    for (uint64_t k = 0; k < C; k++) {
+      uint32_t code = 0;
+      uint64_t bit = k * p->bits;
+      for (uint32_t j = 0; j < p->bits; j++, bit++) code |= (uint32_t)((row[bit >> 3] >> (bit & 7)) & 1u) << j;
+      const float t = (float)((int)code - Lq) * s;
+      const float g = t / c;
+      if (p->dtype) ((uint16_t *)out)[r * C + k] = f32_to_bf16(g);
+      else ((float *)out)[r * C + k] = g;
+    }
+  }
+  return 0;
+}

@@ -726,9 +726,9 @@ __global__ void __launch_bounds__(kThreads, 2) decode_stream_kernel(const Args a
     for (int i = 0; i < C::CPR; ++i) {
       const int piece = i * 32 + lane, r = piece / C::CPR, q = piece % C::CPR;
       const uint64_t t = tile_of(r);
-      if ((rows >> r) & 1u)
-        *reinterpret_cast<uint4 *>(a.out + t * (uint64_t)C::ROWB + (size_t)q * 16) =
-            *reinterpret_cast<const uint4 *>(ostage + (size_t)phys_chunk<C>(r, q) * 16);
+      if ((rows >> r) & 1u)   // streaming store: the tensor is not read again by this library
+        __stcs(reinterpret_cast<uint4 *>(a.out + t * (uint64_t)C::ROWB + (size_t)q * 16),
+               *reinterpret_cast<const uint4 *>(ostage + (size_t)phys_chunk<C>(r, q) * 16));
     }
     __syncwarp();
   };

@@ -1,0 +1,108 @@
+"""Pins of the fixed-point gradient compressor's oracle (Algorithm 1 line 6; appendix "Gradient scaling").
+
+The paper prints no formula for Q_Naive, so the oracle is pinned to what the mathematics fixes: the textbook
+symmetric fixed-point expression (written here independently, in float64), the half-step error bound, sign
+antisymmetry, exact invariance under a power-of-two pre-scale, zero rows, and an independent reader of the
+byte format."""
+import numpy as np
+import pytest
+
+import oracle as O
+
+
+def _grad(shape, seed, scale=1e-3):
+    return (np.random.default_rng(seed).standard_normal(shape) * scale).astype(np.float32)
+
+
+def _read(p: O.QNaiveParams, buf: np.ndarray):
+    """Independent reader of the packed format: (scales, signed codes)."""
+    assert bytes(buf[:4]) == b"TAHN" and int(buf[4:8].view(np.uint32)[0]) == 1
+    assert int(buf[12:16].view(np.uint32)[0]) == p.bits and int(buf[24:28].view(np.uint32)[0]) == p.hidden
+    n_s = 1 if p.per_tensor else p.tokens
+    off_pay = (128 + 4 * n_s + 127) // 128 * 128
+    row_bytes = ((p.hidden * p.bits + 7) // 8 + 15) // 16 * 16
+    scales = buf[128:128 + 4 * n_s].view(np.float32).copy()
+    bits = np.unpackbits(buf[off_pay:off_pay + p.tokens * row_bytes].reshape(p.tokens, row_bytes), axis=1,
+                         bitorder="little")[:, :p.hidden * p.bits].reshape(p.tokens, p.hidden, p.bits)
+    codes = (bits.astype(np.int64) << np.arange(p.bits)).sum(axis=2)
+    return scales, codes - (2 ** (p.bits - 1) - 1), buf[off_pay + p.tokens * row_bytes:]
+
+
+@pytest.mark.parametrize("bits", [2, 4, 6, 8, 10, 16])
+@pytest.mark.parametrize("per_tensor", [0, 1])
+def test_codes_equal_the_textbook_expression(bits, per_tensor):
+    x = _grad((24, 64), bits)
+    x[3] = 0.0                                     # a zero row
+    p = O.QNaiveParams(tokens=24, hidden=64, bits=bits, per_tensor=per_tensor, prescale=1.0)
+    buf = O.qnaive_encode(p, x)
+    scales, q, tail = _read(p, buf)
+    assert not tail.any()                          # padding is zero
+    L = 2 ** (bits - 1) - 1
+    m = np.abs(x).max() * np.ones(24, np.float32) if per_tensor else np.abs(x).max(axis=1)
+    s = (m / np.float32(L)).astype(np.float32)
+    assert np.array_equal(scales, s[:1] if per_tensor else s)
+    inv = np.where(s > 0, np.float32(1) / np.where(s > 0, s, 1).astype(np.float32), np.float32(0)).astype(np.float32)
+    want = np.clip(np.rint(x.astype(np.float64) * inv.astype(np.float64)[:, None]), -L, L).astype(np.int64)
+    assert np.array_equal(q, want)
+    assert np.abs(q).max() <= L and (q[3] == 0).all()
+    # decode: (q * s) / c in binary32; error at most half a step
+    y = O.qnaive_decode(p, buf)
+    assert np.array_equal(y, (q.astype(np.float32) * s[:, None]).astype(np.float32))
+    assert (np.abs(y - x) <= 0.5 * s[:, None] * (1 + 1e-6) + 1e-45).all()
+
+
+def test_sign_antisymmetry_and_extremes():
+    x = _grad((8, 32), 3)
+    p = O.QNaiveParams(tokens=8, hidden=32, bits=6)
+    a = O.qnaive_decode(p, O.qnaive_encode(p, x))
+    b = O.qnaive_decode(p, O.qnaive_encode(p, -x))
+    assert np.array_equal(a, -b)
+    # the row's largest magnitude maps to +-L exactly and comes back as itself up to one rounding
+    _, q, _ = _read(p, O.qnaive_encode(p, x))
+    assert (np.abs(q).max(axis=1) == 31).all()
+    i = np.abs(x).argmax(axis=1)
+    assert np.allclose(a[np.arange(8), i], x[np.arange(8), i], rtol=3e-7)
+
+
+@pytest.mark.parametrize("c", [2.0 ** 10, 2.0 ** -3, 1024.0 * 64])
+def test_power_of_two_prescale_changes_nothing(c):
+    """g_hat = Q(c g) / c: for c a power of two every step scales exactly, so the codes and the decoded
+    values do not depend on c (the pre-scale only matters where c g leaves the subnormal range)."""
+    x = _grad((16, 64), 5, scale=1e-5)
+    p1 = O.QNaiveParams(tokens=16, hidden=64, bits=8, prescale=1.0)
+    pc = O.QNaiveParams(tokens=16, hidden=64, bits=8, prescale=c)
+    b1, bc = O.qnaive_encode(p1, x), O.qnaive_encode(pc, x)
+    assert np.array_equal(_read(p1, b1)[1], _read(pc, bc)[1])
+    assert np.array_equal(O.qnaive_decode(p1, b1), O.qnaive_decode(pc, bc))
+
+
+def test_prescale_rescues_tiny_gradients():
+    """Gradients near the bottom of binary32 lose their scale to underflow; a pre-scale brings them back."""
+    x = _grad((4, 64), 6, scale=1e-41)
+    p1 = O.QNaiveParams(tokens=4, hidden=64, bits=8, prescale=1.0)
+    pc = O.QNaiveParams(tokens=4, hidden=64, bits=8, prescale=2.0 ** 60)
+    e1 = np.abs(O.qnaive_decode(p1, O.qnaive_encode(p1, x)).astype(np.float64) - x).max()
+    ec = np.abs(O.qnaive_decode(pc, O.qnaive_encode(pc, x)).astype(np.float64) - x).max()
+    assert ec < e1
+
+
+def test_bf16_is_widened_binary32_and_error_shrinks_with_bits():
+    import torch
+    x = torch.from_numpy(_grad((8, 128), 9)).to(torch.bfloat16)
+    xb = x.view(torch.int16).numpy().view(np.uint16)
+    xf = x.to(torch.float32).numpy()
+    errs = []
+    for bits in (4, 6, 8, 10):
+        pb = O.QNaiveParams(tokens=8, hidden=128, dtype=O.BF16, bits=bits)
+        pf = O.QNaiveParams(tokens=8, hidden=128, dtype=O.F32, bits=bits)
+        bb, bf = O.qnaive_encode(pb, xb), O.qnaive_encode(pf, xf)
+        assert np.array_equal(bb[128:], bf[128:])                 # same scales and codes
+        errs.append(np.abs(O.qnaive_decode(pf, bf) - xf).max())
+    assert errs == sorted(errs, reverse=True)
+
+
+def test_invalid_parameters():
+    for kw in (dict(bits=1), dict(bits=17), dict(hidden=60), dict(prescale=0.0), dict(prescale=float("inf")),
+               dict(tokens=0), dict(per_tensor=2)):
+        p = O.QNaiveParams(**{**dict(tokens=4, hidden=64), **kw})
+        assert O.qnaive_packed_bound(p) == 0
