@@ -274,6 +274,35 @@ def main():
     e2e_steps = max(3, min(args.steps, 20))
     ms_e2e = timed(e2e_step, e2e_steps)
 
+    # the backward half of the boundary (Algorithm 1 lines 6-7): 6-bit fixed-point gradient compressor,
+    # same shape, gradient-sized values; reported beside the headline, not part of it
+    qn = None
+    if rank == 0:
+        gx = [(x.float() * 1e-4).to(x.dtype) for x in xs]
+        qp = T.QNaiveParams(tokens=w.tokens, hidden=w.hidden, dtype=p.dtype, bits=6, per_tensor=0, prescale=1024.0)
+        qpk = [torch.empty(T.qnaive_packed_bound(qp), dtype=torch.uint8, device=dev) for _ in range(n_sets)]
+        qws = torch.empty(T.qnaive_workspace_bound(qp), dtype=torch.uint8, device=dev)
+
+        def q_rt(i):
+            k = i % n_sets
+            T.qnaive_encode(qp, gx[k], packed=qpk[k], ws=qws)
+            T.qnaive_decode(qp, qpk[k], out=outs[k], ws=qws)
+
+        for i in range(3):
+            q_rt(i)
+        qsteps = max(3, min(args.steps, 50))
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record(stream)
+        for i in range(qsteps):
+            q_rt(i)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        q_ms = e0.elapsed_time(e1) / qsteps
+        q_bytes = 2 * (in_bytes + qpk[0].numel())
+        qn = {"bits": 6, "us": 1e3 * q_ms, "uncompressed_GBps": in_bytes / (q_ms * 1e-3) / 1e9,
+              "hbm_GBps": q_bytes / (q_ms * 1e-3) / 1e9}
+
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -309,6 +338,9 @@ def main():
         path[nm] = {"uncompressed_GBps": gb(in_bytes, ms, args.steps), "us": 1e3 * ms / args.steps,
                     "hbm_GBps": a, "frac_of_measured": a / peak, "frac_of_8TBps": a / 8000.0}
     a = gb(2 * alg_dir, ms_total, args.steps)
+    if qn:
+        qn["frac_of_measured"] = qn["hbm_GBps"] / peak
+        path["backward_qnaive_roundtrip"] = qn
     path["roundtrip"] = {"uncompressed_GBps": value / world, "us": 1e3 * ms_total / args.steps, "hbm_GBps": a,
                          "frac_of_measured": a / peak, "frac_of_8TBps": a / 8000.0}
 

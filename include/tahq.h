@@ -168,6 +168,37 @@ tahq_status tahq_decode(const tahq_params *p, const void *d_packed, size_t packe
 tahq_status tahq_encode_noalloc(const tahq_params *p, const void *d_in, void *d_packed, size_t packed_cap,
                                 tahq_stream stream);
 
+/*
+ * Fixed-point gradient compressor Q_Naive (Algorithm 1 lines 6-7, Sec. 3.5; pre-scale of the appendix,
+ * g_hat = Q(c g) / c).  The paper names it and gives no formula; this library's reading:
+ *   y = c * g (binary32);  per token (row) or per tensor: s = max|y| / L, L = 2^(b-1) - 1, kept as binary32;
+ *   q = clamp(round(y * (1/s)), -L, L), product rounded once, ties to even; code = q + L in b bits;
+ *   g_hat = (q * s) / c (binary32 product, then binary32 division).
+ * Packed buffer: 128-byte header, binary32 scales, then one row of codes per token (little-endian bit
+ * stream, element k at bits [k b, (k+1) b)), rows padded to 16 bytes, sections to 128; size depends on
+ * the parameters only; every byte is written.
+ * d_in / d_out: dense row-major [tokens x hidden] (dtype), device, 16-byte aligned.  d_ws: at least
+ * tahq_qnaive_workspace_bound() bytes; its first 4 bytes are the device status word (TAHQ_DEV_BAD_HEADER
+ * when decode is handed a buffer whose header does not match; the output is then untouched).
+ * Errors as for tahq_encode / tahq_decode.
+ */
+typedef struct {
+  uint32_t struct_size;      /* = sizeof(tahq_qnaive_params)                     */
+  uint32_t dtype;            /* tahq_dtype                                       */
+  uint64_t tokens;
+  uint32_t hidden;           /* a multiple of 8                                  */
+  uint32_t bits;             /* b in [2, 16] (the paper uses 6, 8 and 10)        */
+  uint32_t per_tensor;       /* 0: one scale per token; 1: one for the tensor    */
+  float prescale;            /* c > 0, finite (1.0f = none)                      */
+} tahq_qnaive_params;
+
+size_t tahq_qnaive_packed_bound(const tahq_qnaive_params *p);      /* 0 if the parameters are invalid */
+size_t tahq_qnaive_workspace_bound(const tahq_qnaive_params *p);
+tahq_status tahq_qnaive_encode(const tahq_qnaive_params *p, const void *d_in, void *d_packed, size_t packed_cap,
+                               void *d_ws, size_t ws_cap, tahq_stream stream);
+tahq_status tahq_qnaive_decode(const tahq_qnaive_params *p, const void *d_packed, size_t packed_bytes, void *d_out,
+                               void *d_ws, size_t ws_cap, tahq_stream stream);
+
 /* Static string for a status code. */
 const char *tahq_status_string(tahq_status s);
 

@@ -66,8 +66,30 @@ class TahqError(RuntimeError):
         super().__init__(f"tahq: {status_string(code)} ({code})")
 
 
+class _QParams(C.Structure):
+    _fields_ = [("struct_size", C.c_uint32), ("dtype", C.c_uint32), ("tokens", C.c_uint64), ("hidden", C.c_uint32),
+                ("bits", C.c_uint32), ("per_tensor", C.c_uint32), ("prescale", C.c_float)]
+
+
+@dataclass
+class QNaiveParams:
+    """Fixed-point gradient compressor (Algorithm 1 line 6): b bits, per-token or per-tensor scale, pre-scale c."""
+
+    tokens: int
+    hidden: int
+    dtype: int = F32
+    bits: int = 8
+    per_tensor: int = 0
+    prescale: float = 1.0
+
+    def c(self) -> _QParams:
+        return _QParams(C.sizeof(_QParams), self.dtype, self.tokens, self.hidden, self.bits, self.per_tensor,
+                        self.prescale)
+
+
 EXPORTS = ["tahq_packed_bound", "tahq_packed_layout", "tahq_workspace_bound", "tahq_encode", "tahq_decode",
            "tahq_encode_noalloc",
+           "tahq_qnaive_packed_bound", "tahq_qnaive_workspace_bound", "tahq_qnaive_encode", "tahq_qnaive_decode",
            "tahq_status_string", "tahq_last_launch_count", "tahq_profile", "tahq_profile_read"]
 
 _lib = None
@@ -101,6 +123,15 @@ def lib() -> C.CDLL:
         L.tahq_profile.restype = None
         L.tahq_profile_read.argtypes = [C.c_char_p, C.POINTER(C.c_float), C.c_int]
         L.tahq_profile_read.restype = C.c_int
+        qp = C.POINTER(_QParams)
+        L.tahq_qnaive_packed_bound.argtypes = [qp]
+        L.tahq_qnaive_packed_bound.restype = C.c_size_t
+        L.tahq_qnaive_workspace_bound.argtypes = [qp]
+        L.tahq_qnaive_workspace_bound.restype = C.c_size_t
+        L.tahq_qnaive_encode.argtypes = [qp, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p, C.c_size_t, C.c_void_p]
+        L.tahq_qnaive_encode.restype = C.c_int
+        L.tahq_qnaive_decode.argtypes = [qp, C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+        L.tahq_qnaive_decode.restype = C.c_int
         _lib = L
     return _lib
 
@@ -221,3 +252,45 @@ def decode(p: Params, packed: torch.Tensor, out: torch.Tensor | None = None, ws:
 def device_status(ws: torch.Tensor) -> int:
     """Device status word of the last call that used this workspace (synchronises)."""
     return int(ws[:4].view(torch.int32).item())
+
+
+# ---------------------------------------------------------------- fixed-point gradient compressor
+def qnaive_packed_bound(p: QNaiveParams) -> int:
+    return int(lib().tahq_qnaive_packed_bound(C.byref(p.c())))
+
+
+def qnaive_workspace_bound(p: QNaiveParams) -> int:
+    return int(lib().tahq_qnaive_workspace_bound(C.byref(p.c())))
+
+
+def tahq_qnaive_encode(p: QNaiveParams, d_in: int, d_packed: int, cap: int, d_ws: int, ws_cap: int, stream: int) -> int:
+    return int(lib().tahq_qnaive_encode(C.byref(p.c()), d_in, d_packed, cap, d_ws, ws_cap, stream))
+
+
+def tahq_qnaive_decode(p: QNaiveParams, d_packed: int, nbytes: int, d_out: int, d_ws: int, ws_cap: int, stream: int) -> int:
+    return int(lib().tahq_qnaive_decode(C.byref(p.c()), d_packed, nbytes, d_out, d_ws, ws_cap, stream))
+
+
+def qnaive_encode(p: QNaiveParams, x: torch.Tensor, packed: torch.Tensor | None = None, ws: torch.Tensor | None = None):
+    if packed is None:
+        packed = torch.empty(qnaive_packed_bound(p), dtype=torch.uint8, device=x.device)
+    if ws is None:
+        ws = torch.empty(qnaive_workspace_bound(p), dtype=torch.uint8, device=x.device)
+    rc = tahq_qnaive_encode(p, x.data_ptr(), packed.data_ptr(), packed.numel(), ws.data_ptr(), ws.numel(),
+                            int(torch.cuda.current_stream(x.device).cuda_stream))
+    if rc:
+        raise TahqError(rc)
+    return packed, ws
+
+
+def qnaive_decode(p: QNaiveParams, packed: torch.Tensor, out: torch.Tensor | None = None, ws: torch.Tensor | None = None):
+    if out is None:
+        out = torch.empty((p.tokens, p.hidden), device=packed.device,
+                          dtype=torch.float32 if p.dtype == F32 else torch.bfloat16)
+    if ws is None:
+        ws = torch.empty(qnaive_workspace_bound(p), dtype=torch.uint8, device=packed.device)
+    rc = tahq_qnaive_decode(p, packed.data_ptr(), packed.numel(), out.data_ptr(), ws.data_ptr(), ws.numel(),
+                            int(torch.cuda.current_stream(packed.device).cuda_stream))
+    if rc:
+        raise TahqError(rc)
+    return out, ws

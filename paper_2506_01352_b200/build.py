@@ -8,7 +8,7 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 _CSRC = os.path.join(_PKG, "csrc")
 LIB = os.path.join(_PKG, "libtahq.so")
 SOURCES = [os.path.join(_CSRC, "tahq_api.cu")]
-_DEPS = [os.path.join(_CSRC, f) for f in ("tahq_api.cu", "tahq_kernels.cuh", "tahq_stream.cuh", "tahq_device.cuh")] + [
+_DEPS = [os.path.join(_CSRC, f) for f in ("tahq_api.cu", "tahq_kernels.cuh", "tahq_stream.cuh", "tahq_device.cuh", "qnaive.cuh")] + [
     os.path.join(os.path.dirname(_PKG), "include", "tahq.h")]
 
 NVCC_FLAGS = [

@@ -1,0 +1,281 @@
+// Fixed-point gradient compressor Q_Naive (Algorithm 1 lines 6-7; pre-scale g_hat = Q(c g) / c of
+// the appendix) for sm_100a.  One warp owns one token (row) at a time: a first pass finds the row's
+// largest |c g| (per-tensor scale: a small kernel finds the tensor's beforehand), a second pass --
+// the row is still in L1/L2 -- turns eight consecutive elements per lane into b bytes of codes.
+//   y = c * g;  s = max|y| / (2^(b-1) - 1);  q = clamp(round(y * (1/s)), -L, L);  code = q + L
+// with the product y * (1/s) rounded once (fused multiply-add with 1.5 * 2^23 as the addend).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace tahq {
+
+struct QArgs {
+  const uint8_t *in;      // encode: tensor
+  uint8_t *packed;
+  uint8_t *out;           // decode: tensor
+  uint64_t tokens;
+  uint32_t hidden, bits, per_tensor;
+  float prescale;
+  uint64_t off_scales, off_payload, row_bytes, total_bytes;
+  uint32_t *gmax;         // per-tensor mode: bits of max |c g| (zeroed per call)
+  uint32_t *status;
+  uint32_t header[16];
+};
+
+constexpr int kQThreads = 256;
+constexpr float kQMagic = 12582912.0f;   // 1.5 * 2^23
+
+// eight consecutive elements, widened to binary32
+template <bool BF16>
+__device__ __forceinline__ void q_load8(const uint8_t *row, uint32_t k0, float (&v)[8]) {
+  if constexpr (BF16) {
+    const uint4 w = __ldg(reinterpret_cast<const uint4 *>(row + (size_t)k0 * 2));
+    const uint32_t u[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      v[2 * j] = __uint_as_float(u[j] << 16);
+      v[2 * j + 1] = __uint_as_float(u[j] & 0xffff0000u);
+    }
+  } else {
+    const float4 a = __ldg(reinterpret_cast<const float4 *>(row + (size_t)k0 * 4));
+    const float4 b = __ldg(reinterpret_cast<const float4 *>(row + (size_t)k0 * 4) + 1);
+    v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w;
+    v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+  }
+}
+
+__device__ __forceinline__ float warp_max(float m) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+  return m;
+}
+
+// per-tensor mode: max |c g| over the whole tensor (non-negative floats order like their bit patterns)
+template <bool BF16>
+__global__ void __launch_bounds__(kQThreads) qnaive_max_kernel(const QArgs a) {
+  const uint64_t n8 = a.tokens * (uint64_t)(a.hidden / 8);
+  float m = 0.0f;
+  for (uint64_t i = (uint64_t)blockIdx.x * kQThreads + threadIdx.x; i < n8; i += (uint64_t)gridDim.x * kQThreads) {
+    float v[8];
+    q_load8<BF16>(a.in + i * (uint64_t)(BF16 ? 16 : 32), 0, v);
+#pragma unroll
+    for (int k = 0; k < 8; ++k) m = fmaxf(m, fabsf(a.prescale * v[k]));
+  }
+  m = warp_max(m);
+  if ((threadIdx.x & 31) == 0 && m > 0.0f) atomicMax(a.gmax, __float_as_uint(m));
+}
+
+template <bool BF16>
+__global__ void __launch_bounds__(kQThreads, 2) qnaive_encode_kernel(const QArgs a) {
+  constexpr int ESZ = BF16 ? 2 : 4;
+  const int lane = threadIdx.x & 31;
+  const uint64_t warp = ((uint64_t)blockIdx.x * kQThreads + threadIdx.x) >> 5;
+  const uint64_t n_warps = ((uint64_t)gridDim.x * kQThreads) >> 5;
+  const uint32_t b = a.bits, C = a.hidden;
+  const int Lq = (int)((1u << (b - 1)) - 1u);
+  const float Lf = (float)Lq;
+  float *scales = reinterpret_cast<float *>(a.packed + a.off_scales);
+
+  if (blockIdx.x == 0) {   // header and section padding
+    if (threadIdx.x < 32) reinterpret_cast<uint32_t *>(a.packed)[threadIdx.x] = threadIdx.x < 16 ? a.header[threadIdx.x] : 0u;
+    const uint64_t n_s = a.per_tensor ? 1 : a.tokens;
+    for (uint64_t o = a.off_scales + 4 * n_s + threadIdx.x; o < a.off_payload; o += kQThreads) a.packed[o] = 0;
+    for (uint64_t o = a.off_payload + a.tokens * a.row_bytes + threadIdx.x; o < a.total_bytes; o += kQThreads) a.packed[o] = 0;
+  }
+  const uint32_t data_bytes = (uint32_t)(((uint64_t)C * b) >> 3);   // hidden is a multiple of 8
+  // pieces a lane's b bytes are stored in: the largest power of two dividing b, at most 16
+  const uint32_t gsz = (b & (0u - b)) > 16u ? 16u : (b & (0u - b));
+
+  // one group of eight elements -> the lane's b bytes of codes at dst
+  auto emit = [&](const float (&v)[8], float inv, uint8_t *dst) {
+    unsigned long long lo = 0, hi = 0;   // b bytes as a 128-bit little-endian value
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+      const float y = a.prescale * v[k];
+      const float t = __fmaf_rn(y, inv, kQMagic);   // one rounding, ties to even
+      int q = (int)(__float_as_uint(t) - 0x4B400000u);
+      q = min(max(q, -Lq), Lq);
+      const unsigned long long code = (unsigned long long)(uint32_t)(q + Lq);
+      const uint32_t pos = (uint32_t)k * b;
+      if (pos < 64) {
+        lo |= code << pos;
+        if (pos + b > 64) hi |= code >> (64 - pos);
+      } else {
+        hi |= code << (pos - 64);
+      }
+    }
+    if (gsz == 16) {
+      *reinterpret_cast<uint4 *>(dst) = make_uint4((uint32_t)lo, (uint32_t)(lo >> 32), (uint32_t)hi, (uint32_t)(hi >> 32));
+    } else if (gsz == 8) {
+      *reinterpret_cast<unsigned long long *>(dst) = lo;
+    } else if (gsz == 4) {
+#pragma unroll
+      for (int j = 0; j < 3; ++j)
+        if ((uint32_t)(4 * j) < b) reinterpret_cast<uint32_t *>(dst)[j] = (uint32_t)(j < 2 ? lo >> (32 * j) : hi);
+    } else if (gsz == 2) {
+#pragma unroll
+      for (int j = 0; j < 7; ++j)
+        if ((uint32_t)(2 * j) < b)
+          reinterpret_cast<uint16_t *>(dst)[j] = (uint16_t)(j < 4 ? lo >> (16 * j) : hi >> (16 * (j - 4)));
+    } else {
+#pragma unroll
+      for (int j = 0; j < 15; ++j)
+        if ((uint32_t)j < b) dst[j] = (uint8_t)(j < 8 ? lo >> (8 * j) : hi >> (8 * (j - 8)));
+    }
+  };
+  constexpr int kHeld = BF16 ? 16 : 8;   // groups of eight elements a lane keeps in registers (64 registers)
+  const bool held = C <= (uint32_t)kHeld * 256u;
+
+  for (uint64_t r = warp; r < a.tokens; r += n_warps) {
+    const uint8_t *row = a.in + r * (uint64_t)C * ESZ;
+    uint8_t *orow = a.packed + a.off_payload + r * a.row_bytes;
+    float m = 0.0f;
+    if (held) {   // the row is read once: all loads in flight together, then the range, then the codes
+      uint4 raw[kHeld][BF16 ? 1 : 2];   // as loaded; widened where used
+#pragma unroll
+      for (int i = 0; i < kHeld; ++i) {
+        const uint32_t k0 = (uint32_t)i * 256u + lane * 8;
+#pragma unroll
+        for (int h = 0; h < (BF16 ? 1 : 2); ++h)
+          raw[i][h] = k0 < C ? __ldg(reinterpret_cast<const uint4 *>(row + (size_t)k0 * ESZ) + h) : make_uint4(0, 0, 0, 0);
+      }
+      auto widen = [&](int i, float (&v)[8]) {
+        if constexpr (BF16) {
+          const uint32_t u[4] = {raw[i][0].x, raw[i][0].y, raw[i][0].z, raw[i][0].w};
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            v[2 * j] = __uint_as_float(u[j] << 16);
+            v[2 * j + 1] = __uint_as_float(u[j] & 0xffff0000u);
+          }
+        } else {
+          const uint32_t u[8] = {raw[i][0].x, raw[i][0].y, raw[i][0].z, raw[i][0].w,
+                                 raw[i][BF16 ? 0 : 1].x, raw[i][BF16 ? 0 : 1].y, raw[i][BF16 ? 0 : 1].z, raw[i][BF16 ? 0 : 1].w};
+#pragma unroll
+          for (int j = 0; j < 8; ++j) v[j] = __uint_as_float(u[j]);
+        }
+      };
+      if (a.per_tensor) {
+        m = __uint_as_float(*a.gmax);
+      } else {
+#pragma unroll
+        for (int i = 0; i < kHeld; ++i) {
+          float v[8];
+          widen(i, v);
+#pragma unroll
+          for (int k = 0; k < 8; ++k) m = fmaxf(m, fabsf(a.prescale * v[k]));
+        }
+        m = warp_max(m);
+      }
+      const float s = __fdiv_rn(m, Lf);
+      const float inv = s > 0.0f ? __frcp_rn(s) : 0.0f;
+      if (lane == 0 && (!a.per_tensor || r == 0)) scales[a.per_tensor ? 0 : r] = s;
+#pragma unroll
+      for (int i = 0; i < kHeld; ++i) {
+        const uint32_t k0 = (uint32_t)i * 256u + lane * 8;
+        if (k0 < C) {
+          float v[8];
+          widen(i, v);
+          emit(v, inv, orow + (size_t)(k0 >> 3) * b);
+        }
+      }
+    } else {      // long rows: a pass for the range, a second one (from L1/L2) for the codes
+      if (a.per_tensor) {
+        m = __uint_as_float(*a.gmax);
+      } else {
+#pragma unroll 4
+        for (uint32_t k0 = lane * 8; k0 < C; k0 += 256) {
+          float v[8];
+          q_load8<BF16>(row, k0, v);
+#pragma unroll
+          for (int k = 0; k < 8; ++k) m = fmaxf(m, fabsf(a.prescale * v[k]));
+        }
+        m = warp_max(m);
+      }
+      const float s = __fdiv_rn(m, Lf);
+      const float inv = s > 0.0f ? __frcp_rn(s) : 0.0f;
+      if (lane == 0 && (!a.per_tensor || r == 0)) scales[a.per_tensor ? 0 : r] = s;
+#pragma unroll 2
+      for (uint32_t k0 = lane * 8; k0 < C; k0 += 256) {
+        float v[8];
+        q_load8<BF16>(row, k0, v);
+        emit(v, inv, orow + (size_t)(k0 >> 3) * b);
+      }
+    }
+    for (uint32_t o = data_bytes + lane; o < (uint32_t)a.row_bytes; o += 32) orow[o] = 0;   // the row's padding
+  }
+}
+
+template <bool BF16>
+__global__ void __launch_bounds__(kQThreads) qnaive_decode_kernel(const QArgs a) {
+  constexpr int ESZ = BF16 ? 2 : 4;
+  const int lane = threadIdx.x & 31;
+  const uint64_t warp = ((uint64_t)blockIdx.x * kQThreads + threadIdx.x) >> 5;
+  const uint64_t n_warps = ((uint64_t)gridDim.x * kQThreads) >> 5;
+  const uint32_t b = a.bits, C = a.hidden;
+  const int Lq = (int)((1u << (b - 1)) - 1u);
+  // the received header must describe these parameters; otherwise nothing is written
+  {
+    const uint32_t w = lane < 16 ? __ldg(reinterpret_cast<const uint32_t *>(a.packed) + lane) : 0u;
+    const bool bad = lane < 16 && w != a.header[lane];
+    if (__any_sync(0xffffffffu, bad)) {
+      if (blockIdx.x == 0 && threadIdx.x == 0) atomicOr(a.status, 1u /* TAHQ_DEV_BAD_HEADER */);
+      return;
+    }
+  }
+  const float *scales = reinterpret_cast<const float *>(a.packed + a.off_scales);
+  const unsigned long long mask = (1ull << b) - 1ull;
+  // dividing by a power of two is the same rounding as multiplying by its (exact) reciprocal
+  const bool pow2 = (__float_as_uint(a.prescale) & 0x007fffffu) == 0u && (__float_as_uint(a.prescale) >> 23) - 2u < 250u;
+  const float rc = pow2 ? __frcp_rn(a.prescale) : 0.0f;
+  for (uint64_t r = warp; r < a.tokens; r += n_warps) {
+    const float s = __ldg(scales + (a.per_tensor ? 0 : r));
+    const uint8_t *irow = a.packed + a.off_payload + r * a.row_bytes;
+    uint8_t *orow = a.out + r * (uint64_t)C * ESZ;
+#pragma unroll 4
+    for (uint32_t k0 = lane * 8; k0 < C; k0 += 256) {
+      // the lane's b bytes start at byte o of the row; fetch the five aligned words that cover them
+      const uint32_t o = (k0 >> 3) * b, o4 = o & ~3u, sh = (o & 3u) * 8u;
+      uint32_t w[5];
+#pragma unroll
+      for (int j = 0; j < 5; ++j)
+        w[j] = (o4 + 4u * j < (uint32_t)a.row_bytes) ? __ldg(reinterpret_cast<const uint32_t *>(irow + o4) + j) : 0u;
+      uint32_t x[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) x[j] = __funnelshift_r(w[j], w[j + 1], sh);
+      const unsigned long long lo = (unsigned long long)x[0] | ((unsigned long long)x[1] << 32);
+      const unsigned long long hi = (unsigned long long)x[2] | ((unsigned long long)x[3] << 32);
+      float g[8];
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        const uint32_t pos = (uint32_t)k * b;
+        unsigned long long c;
+        if (pos < 64) {
+          c = lo >> pos;
+          if (pos + b > 64) c |= hi << (64 - pos);
+        } else {
+          c = hi >> (pos - 64);
+        }
+        const int q = (int)(uint32_t)(c & mask) - Lq;
+        const float t = __fmul_rn((float)q, s);
+        g[k] = pow2 ? __fmul_rn(t, rc) : __fdiv_rn(t, a.prescale);
+      }
+      if constexpr (BF16) {
+        uint32_t u[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const __nv_bfloat162 h2 = __floats2bfloat162_rn(g[2 * j], g[2 * j + 1]);
+          u[j] = *reinterpret_cast<const uint32_t *>(&h2);
+        }
+        *reinterpret_cast<uint4 *>(orow + (size_t)k0 * 2) = make_uint4(u[0], u[1], u[2], u[3]);
+      } else {
+        reinterpret_cast<float4 *>(orow + (size_t)k0 * 4)[0] = make_float4(g[0], g[1], g[2], g[3]);
+        reinterpret_cast<float4 *>(orow + (size_t)k0 * 4)[1] = make_float4(g[4], g[5], g[6], g[7]);
+      }
+    }
+  }
+}
+
+}  // namespace tahq

@@ -7,6 +7,7 @@
 #include <vector>
 
 #include "tahq_stream.cuh"
+#include "qnaive.cuh"
 
 namespace tahq {
 
@@ -380,6 +381,103 @@ tahq_status tahq_encode_noalloc(const tahq_params *p, const void *d_in, void *d_
   }
   // tahq_encode clears the head of the workspace (status, flags, histograms, counters) on the stream
   return tahq_encode(p, d_in, d_packed, packed_cap, g_noalloc_addr[dev], TAHQ_NOALLOC_SCRATCH_BYTES, stream);
+}
+
+// ---- fixed-point gradient compressor -------------------------------------------------------------------
+namespace {
+struct QPlan { uint64_t n_scales, off_scales, off_payload, row_bytes, total_bytes; };
+tahq_status q_plan(const tahq_qnaive_params *p, QPlan *q) {
+  if (!p || p->struct_size != sizeof(tahq_qnaive_params)) return TAHQ_ERR_INVALID_ARG;
+  if (p->dtype > 1 || p->per_tensor > 1) return TAHQ_ERR_INVALID_ARG;
+  if (p->tokens == 0 || p->hidden == 0 || p->hidden % 8) return TAHQ_ERR_INVALID_ARG;
+  if (p->bits < 2 || p->bits > 16) return TAHQ_ERR_INVALID_ARG;
+  if (!(p->prescale > 0.0f) || p->prescale > 3.402823466e38f) return TAHQ_ERR_INVALID_ARG;
+  q->n_scales = p->per_tensor ? 1 : p->tokens;
+  q->row_bytes = up(((uint64_t)p->hidden * p->bits + 7) / 8, 16);
+  q->off_scales = 128;
+  q->off_payload = up(q->off_scales + 4 * q->n_scales, 128);
+  q->total_bytes = up(q->off_payload + p->tokens * q->row_bytes, 128);
+  return TAHQ_OK;
+}
+void q_args(const tahq_qnaive_params *p, const QPlan &q, QArgs *a, void *ws) {
+  std::memset(a, 0, sizeof(*a));
+  a->tokens = p->tokens; a->hidden = p->hidden; a->bits = p->bits; a->per_tensor = p->per_tensor;
+  a->prescale = p->prescale;
+  a->off_scales = q.off_scales; a->off_payload = q.off_payload; a->row_bytes = q.row_bytes; a->total_bytes = q.total_bytes;
+  a->status = reinterpret_cast<uint32_t *>(ws);
+  a->gmax = reinterpret_cast<uint32_t *>(ws) + 16;
+  uint32_t *h = a->header;
+  std::memcpy(h, "TAHN", 4);
+  h[1] = 1; h[2] = p->dtype; h[3] = p->bits;
+  h[4] = (uint32_t)p->tokens; h[5] = (uint32_t)(p->tokens >> 32);
+  h[6] = p->hidden; h[7] = p->per_tensor;
+  std::memcpy(&h[8], &p->prescale, 4);
+  h[10] = (uint32_t)q.row_bytes; h[11] = (uint32_t)(q.row_bytes >> 32);
+  h[12] = (uint32_t)q.total_bytes; h[13] = (uint32_t)(q.total_bytes >> 32);
+}
+unsigned q_grid(uint64_t tokens, const DevInfo &d) {
+  const uint64_t want = (tokens + 7) / 8, cap = (uint64_t)d.sms * 8;
+  return (unsigned)(want < cap ? want : cap);
+}
+}  // namespace
+
+size_t tahq_qnaive_packed_bound(const tahq_qnaive_params *p) {
+  QPlan q;
+  return q_plan(p, &q) == TAHQ_OK ? (size_t)q.total_bytes : 0;
+}
+
+size_t tahq_qnaive_workspace_bound(const tahq_qnaive_params *p) {
+  QPlan q;
+  return q_plan(p, &q) == TAHQ_OK ? 256 : 0;
+}
+
+tahq_status tahq_qnaive_encode(const tahq_qnaive_params *p, const void *d_in, void *d_packed, size_t packed_cap,
+                               void *d_ws, size_t ws_cap, tahq_stream stream) {
+  QPlan q;
+  g_launches = 0;
+  if (tahq_status rc = q_plan(p, &q)) return rc;
+  if (!d_in || !d_packed || !d_ws) return TAHQ_ERR_INVALID_ARG;
+  if (packed_cap < q.total_bytes || ws_cap < 256) return TAHQ_ERR_BUFFER_TOO_SMALL;
+  if (!aligned16(d_in) || !aligned16(d_packed) || !aligned16(d_ws)) return TAHQ_ERR_MISALIGNED;
+  DevInfo d;
+  if (!dev_info(&d)) return TAHQ_ERR_CUDA;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  QArgs a;
+  q_args(p, q, &a, d_ws);
+  a.in = static_cast<const uint8_t *>(d_in);
+  a.packed = static_cast<uint8_t *>(d_packed);
+  if (cudaMemsetAsync(d_ws, 0, 256, st) != cudaSuccess) return TAHQ_ERR_CUDA;
+  const bool bf = p->dtype == TAHQ_BF16;
+  if (p->per_tensor) {
+    if (bf) TAHQ_LAUNCH("qnaive_max", st, qnaive_max_kernel<true><<<d.sms * 4, kQThreads, 0, st>>>(a));
+    else TAHQ_LAUNCH("qnaive_max", st, qnaive_max_kernel<false><<<d.sms * 4, kQThreads, 0, st>>>(a));
+  }
+  if (bf) TAHQ_LAUNCH("qnaive_encode", st, qnaive_encode_kernel<true><<<q_grid(p->tokens, d), kQThreads, 0, st>>>(a));
+  else TAHQ_LAUNCH("qnaive_encode", st, qnaive_encode_kernel<false><<<q_grid(p->tokens, d), kQThreads, 0, st>>>(a));
+  return cudaGetLastError() == cudaSuccess ? TAHQ_OK : TAHQ_ERR_CUDA;
+}
+
+tahq_status tahq_qnaive_decode(const tahq_qnaive_params *p, const void *d_packed, size_t packed_bytes, void *d_out,
+                               void *d_ws, size_t ws_cap, tahq_stream stream) {
+  QPlan q;
+  g_launches = 0;
+  if (tahq_status rc = q_plan(p, &q)) return rc;
+  if (!d_packed || !d_out || !d_ws) return TAHQ_ERR_INVALID_ARG;
+  if (packed_bytes < q.total_bytes || ws_cap < 256) return TAHQ_ERR_BUFFER_TOO_SMALL;
+  if (!aligned16(d_packed) || !aligned16(d_out) || !aligned16(d_ws)) return TAHQ_ERR_MISALIGNED;
+  DevInfo d;
+  if (!dev_info(&d)) return TAHQ_ERR_CUDA;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  QArgs a;
+  q_args(p, q, &a, d_ws);
+  a.packed = const_cast<uint8_t *>(static_cast<const uint8_t *>(d_packed));
+  a.out = static_cast<uint8_t *>(d_out);
+  if (cudaMemsetAsync(d_ws, 0, 256, st) != cudaSuccess) return TAHQ_ERR_CUDA;
+  if (p->dtype == TAHQ_BF16)
+    TAHQ_LAUNCH("qnaive_decode", st, qnaive_decode_kernel<true><<<q_grid(p->tokens, d), kQThreads, 0, st>>>(a));
+  else
+    TAHQ_LAUNCH("qnaive_decode", st, qnaive_decode_kernel<false><<<q_grid(p->tokens, d), kQThreads, 0, st>>>(a));
+  return cudaGetLastError() == cudaSuccess ? TAHQ_OK : TAHQ_ERR_CUDA;
 }
 
 const char *tahq_status_string(tahq_status s) {

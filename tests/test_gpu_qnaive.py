@@ -1,0 +1,67 @@
+"""Parity of the CUDA fixed-point gradient compressor with its CPU oracle, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+import oracle as O
+from paper_2506_01352_b200 import binding as T
+from paper_2506_01352_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+
+def _check(x: torch.Tensor, bits: int, per_tensor: int, c: float):
+    dt = T.F32 if x.dtype == torch.float32 else T.BF16
+    p = T.QNaiveParams(tokens=x.shape[0], hidden=x.shape[1], dtype=dt, bits=bits, per_tensor=per_tensor, prescale=c)
+    po = O.QNaiveParams(tokens=x.shape[0], hidden=x.shape[1], dtype=dt, bits=bits, per_tensor=per_tensor, prescale=c)
+    assert T.qnaive_packed_bound(p) == O.qnaive_packed_bound(po)
+    packed = torch.full((T.qnaive_packed_bound(p),), 0xA5, dtype=torch.uint8, device=x.device)
+    packed, ws = T.qnaive_encode(p, x, packed=packed)
+    torch.cuda.synchronize()
+    assert T.device_status(ws) == 0
+    want = O.qnaive_encode(po, synth.to_host_array(x))
+    got = packed.cpu().numpy()
+    if not np.array_equal(got, want):
+        bad = np.flatnonzero(got != want)
+        raise AssertionError(f"{bad.size} differing bytes, first at {bad[:8]}")
+    out = torch.full_like(x, float("nan"))
+    out, ws = T.qnaive_decode(p, packed, out=out)
+    torch.cuda.synchronize()
+    assert T.device_status(ws) == 0
+    y = synth.to_host_array(out)
+    yo = O.qnaive_decode(po, want)
+    assert np.array_equal(y.view(np.uint32 if dt == T.F32 else np.uint16), yo.view(np.uint32 if dt == T.F32 else np.uint16))
+
+
+@pytest.mark.parametrize("bits", [2, 3, 4, 5, 6, 7, 8, 9, 10, 12, 16])
+@pytest.mark.parametrize("per_tensor", [0, 1])
+def test_gradient_like_tensor(bits, per_tensor):
+    x = synth.make("c2_gpt2s", variant=1, device="cuda")[:1024]          # N(0, 1e-3) gradient stand-in, 1024 x 768
+    _check(x.contiguous(), bits, per_tensor, 1024.0)
+
+
+@pytest.mark.parametrize("shape", [(1, 8), (3, 40), (7, 264), (33, 4096), (2, 8200)])
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_ragged_shapes_and_dtypes(shape, dtype):
+    g = torch.Generator(device="cuda").manual_seed(5)
+    x = (torch.randn(shape, generator=g, device="cuda") * 1e-3).to(dtype)
+    x[0] = 0
+    for bits, c in ((6, 1.0), (10, 3.0), (8, 2.0 ** 20)):
+        _check(x, bits, 0, c)
+    _check(x, 6, 1, 1.0)
+
+
+def test_llama_shaped_gradient_bf16():
+    x = (synth.make("c3_llama7b", device="cuda").float() * 1e-4).to(torch.bfloat16)
+    _check(x, 6, 0, 4096.0)
+
+
+def test_refuses_a_foreign_buffer():
+    x = torch.randn(16, 64, device="cuda")
+    p = T.QNaiveParams(tokens=16, hidden=64, bits=8)
+    packed, _ = T.qnaive_encode(p, x)
+    p2 = T.QNaiveParams(tokens=16, hidden=64, bits=8, prescale=2.0)
+    out = torch.full_like(x, 7.0)
+    out, ws = T.qnaive_decode(p2, packed, out=out)
+    torch.cuda.synchronize()
+    assert T.device_status(ws) & 1 and bool((out == 7.0).all())
