@@ -3,6 +3,7 @@
 #include "../../include/tahq.h"
 
 #include <atomic>
+#include <cstdlib>
 #include <cstring>
 #include <vector>
 
@@ -88,7 +89,8 @@ static tahq_status make_plan(const tahq_params *p, Plan *pl) {
   pl->cand_cap = 0;
   if (pl->mixed && !pl->direct) {
     pl->cpg = (uint32_t)((L.tiles_per_group + kSelSlice - 1) / kSelSlice);
-    pl->cand_cap = (uint32_t)(L.tiles_per_group < 32768 ? L.tiles_per_group : 32768);
+    // every tile of a group can end up a candidate (all scores equal): the list holds them all
+    pl->cand_cap = (uint32_t)(L.tiles_per_group < 0xffffffffull ? L.tiles_per_group : 0xffffffffull);
   }
   const bool hist = pl->mixed && !pl->direct;
   uint64_t o = 256;                                         // status word and friends
@@ -148,6 +150,7 @@ static void fill_args(const tahq_params *p, const Plan &pl, uint8_t *ws, Args *a
   a->seed = p->seed;
   a->eps_ratio = p->eps_ratio;
   a->status = reinterpret_cast<uint32_t *>(ws);
+  a->gbar = reinterpret_cast<uint32_t *>(ws) + 16;   // inside the status block, cleared with it
   a->ncand = reinterpret_cast<uint32_t *>(ws + pl.ws_ncand);
   a->hist = reinterpret_cast<uint32_t *>(ws + pl.ws_hist);
   a->scores = reinterpret_cast<float *>(ws + pl.ws_scores);
@@ -199,12 +202,45 @@ static unsigned persistent_grid(uint64_t n_chunks, const DevInfo &d, int occ) {
   return (unsigned)(n_chunks < cap ? n_chunks : cap);
 }
 
+// TAHQ_ENCODE_PATH=split in the environment keeps encode on the three-kernel path (used by the tests to
+// cover it on devices where the cooperative launch always succeeds).
+static bool split_encode_forced() {
+  static const bool v = [] {
+    const char *e = std::getenv("TAHQ_ENCODE_PATH");
+    return e && std::strcmp(e, "split") == 0;
+  }();
+  return v;
+}
+
 template <class C, bool SR>
 static tahq_status encode_t(const Plan &pl, const Args &a, cudaStream_t st) {
   DevInfo d;
   if (!dev_info(&d)) return TAHQ_ERR_CUDA;
   const uint64_t n_chunks = (a.n_tiles + C::TPC - 1) / C::TPC;
-  static std::atomic<int> occ_stats[64], occ_quant[64], sel_ready[64];
+  static std::atomic<int> occ_stats[64], occ_quant[64], sel_ready[64], occ_fused[64];
+  if constexpr (C::LPT == 1) {
+    // large ranking groups: the whole encode as one cooperative launch (grid-wide barriers between scoring,
+    // the exact re-scoring near each group's threshold, and quantise + pack); if the device cannot keep the
+    // grid resident the three-kernel path below does the same work
+    if (pl.mixed && !pl.direct && !split_encode_forced()) {
+      const int smem = StreamCfg<C>::smem_bytes(2);
+      const int occ = prepare(encode_fused_kernel<C, SR>, smem, d, occ_fused);
+      if (occ) {
+        const uint64_t n_units = (a.n_tiles + 31) / 32;
+        const unsigned grid = persistent_grid((n_units + kWarps - 1) / kWarps, d, occ);
+        void *args[] = {const_cast<Args *>(&a)};
+        cudaError_t e;
+        {
+          LaunchScope scope_("encode_fused", st);
+          e = cudaLaunchCooperativeKernel(reinterpret_cast<void *>(encode_fused_kernel<C, SR>), dim3(grid),
+                                          dim3(kThreads), args, (size_t)smem, st);
+        }
+        if (e == cudaSuccess) return TAHQ_OK;
+        cudaGetLastError();   // not launched: fall through
+        --g_launches;
+      }
+    }
+  }
   if (pl.mixed) {
     if constexpr (C::LPT == 1) {
       constexpr int NS = C::ROWB <= 128 ? 3 : 2;

@@ -36,6 +36,7 @@ struct Args {
   uint32_t direct;          // small groups: select_kernel ranks all scores of the group itself
   uint32_t exact_scores;    // stats_kernel writes exact scores (small groups, or a varsigma too large to screen)
   unsigned long long *flags;// [kMaxGrid] (zeroed per call) per-CTA published counts for the offset prefix
+  uint32_t *gbar;           // [2] (zeroed per call) arrival counters of the fused encode kernel's grid barriers
   uint32_t *status;         // device status word
   unsigned long long seed;  // stochastic rounding mode: the generator's key
   uint32_t header[32];      // the 128-byte header of the packed buffer
@@ -197,7 +198,7 @@ __device__ __forceinline__ unsigned long long radix_select(uint64_t count, uint3
   // bits on which the keys differ: a pass over a digit that is the same in every key is skipped
   __shared__ unsigned long long s_or[kSelThreads / 32], s_and[kSelThreads / 32];
   unsigned long long orv = 0, andv = ~0ull;
-  for (uint64_t i = threadIdx.x; i < count; i += kSelThreads) {
+  for (uint64_t i = threadIdx.x; i < count; i += blockDim.x) {
     unsigned long long key;
     if (get(i, key)) { orv |= key; andv &= key; }
   }
@@ -208,8 +209,7 @@ __device__ __forceinline__ unsigned long long radix_select(uint64_t count, uint3
   }
   if ((threadIdx.x & 31) == 0) { s_or[threadIdx.x >> 5] = orv; s_and[threadIdx.x >> 5] = andv; }
   __syncthreads();
-#pragma unroll
-  for (int w = 0; w < kSelThreads / 32; ++w) { orv |= s_or[w]; andv &= s_and[w]; }
+  for (int w = 0; w < (int)(blockDim.x / 32); ++w) { orv |= s_or[w]; andv &= s_and[w]; }
   const unsigned long long varying = orv ^ andv;
   unsigned long long prefix = 0, mask = 0;
   for (int shift = 56; shift >= 0; shift -= 8) {
@@ -219,7 +219,8 @@ __device__ __forceinline__ unsigned long long radix_select(uint64_t count, uint3
       continue;
     }
     if (threadIdx.x < 256) h[threadIdx.x] = 0;
-    for (uint64_t i = threadIdx.x; i < count; i += kSelThreads) {
+    __syncthreads();   // the digit counts are clear before anyone adds to them
+    for (uint64_t i = threadIdx.x; i < count; i += blockDim.x) {
       unsigned long long key;
       if (get(i, key) && (key & mask) == prefix) atomicAdd(&h[(unsigned)(key >> shift) & 255u], 1u);
     }
@@ -255,9 +256,9 @@ __device__ __forceinline__ unsigned long long radix_select(uint64_t count, uint3
 }
 
 constexpr int kSelSlice = 4 * kSelThreads;   // scores one CTA of select_kernel scans (four per thread, loaded at once)
-// Screening scores differ from exact ones by less than kScreenErr = 2.4e-4 (measured bound on the
-// approximate log2: 1e-5 per term, terms weighted by p with sum p <= 1, plus rounding); the band around
-// the threshold bin is 2*kScreenErr wide on each side, expressed in bins (kBinScale bins per unit).
+// Screening scores differ from exact ones by less than kScreenErr = 1e-4 (see tile_score_screen); the
+// band around the threshold bin reaches 0.25 bin = 4.9e-4 beyond it on each side (kBinScale bins per unit
+// of score), more than twice that error.
 constexpr float kScreenBand = 0.25f;
 
 __global__ void __launch_bounds__(kSelThreads) select_kernel(const Args a) {
@@ -444,11 +445,14 @@ struct GroupCursor {
     rem = (uint32_t)r;
   }
   // is the tile `off` tiles after the cursor among the k_hi highest-ranked of its group?
+  // COH: scores and thresholds were written earlier in the same kernel (no read-only path)
+  template <bool COH = false>
   __device__ __forceinline__ bool is_hi(const Args &a, uint64_t tile, uint32_t off) const {
     uint64_t gg = g;
     uint64_t i = (uint64_t)rem + off;
     if (i >= a.tiles_per_group) { gg += i / a.tiles_per_group; i %= a.tiles_per_group; }
-    return rank_key(__ldg(a.scores + tile), (uint32_t)i) >= __ldg(a.theta + gg);
+    if constexpr (COH) return rank_key(__ldcg(a.scores + tile), (uint32_t)i) >= __ldcg(a.theta + gg);
+    else return rank_key(__ldg(a.scores + tile), (uint32_t)i) >= __ldg(a.theta + gg);
   }
   // the same with the tile's score already at hand
   __device__ __forceinline__ bool is_hi_score(const Args &a, float score, uint32_t off) const {
