@@ -202,12 +202,14 @@ static unsigned persistent_grid(uint64_t n_chunks, const DevInfo &d, int occ) {
   return (unsigned)(n_chunks < cap ? n_chunks : cap);
 }
 
-// TAHQ_ENCODE_PATH=split in the environment keeps encode on the three-kernel path (used by the tests to
-// cover it on devices where the cooperative launch always succeeds).
-static bool split_encode_forced() {
+// TAHQ_ENCODE_PATH=fused in the environment switches large-group encodes to the single cooperative kernel.
+// It is off by default: measured on B200 it never beat the three-kernel path (equal encode time on the
+// LLaMA-7B-shaped tensor, 7 % slower round trips because a cooperative launch does not overlap its
+// neighbours' launch latency; 7-13 % slower on 320 MiB and 1 GiB tensors).
+static bool fused_encode_wanted() {
   static const bool v = [] {
     const char *e = std::getenv("TAHQ_ENCODE_PATH");
-    return e && std::strcmp(e, "split") == 0;
+    return e && std::strcmp(e, "fused") == 0;
   }();
   return v;
 }
@@ -219,10 +221,10 @@ static tahq_status encode_t(const Plan &pl, const Args &a, cudaStream_t st) {
   const uint64_t n_chunks = (a.n_tiles + C::TPC - 1) / C::TPC;
   static std::atomic<int> occ_stats[64], occ_quant[64], sel_ready[64], occ_fused[64];
   if constexpr (C::LPT == 1) {
-    // large ranking groups: the whole encode as one cooperative launch (grid-wide barriers between scoring,
-    // the exact re-scoring near each group's threshold, and quantise + pack); if the device cannot keep the
-    // grid resident the three-kernel path below does the same work
-    if (pl.mixed && !pl.direct && !split_encode_forced()) {
+    // large ranking groups, on request: the whole encode as one cooperative launch (grid-wide barriers
+    // between scoring, the exact re-scoring near each group's threshold, and quantise + pack); if the device
+    // cannot keep the grid resident the three-kernel path below does the same work
+    if (pl.mixed && !pl.direct && fused_encode_wanted()) {
       const int smem = StreamCfg<C>::smem_bytes(2);
       const int occ = prepare(encode_fused_kernel<C, SR>, smem, d, occ_fused);
       if (occ) {
