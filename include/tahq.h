@@ -199,6 +199,15 @@ tahq_status tahq_qnaive_encode(const tahq_qnaive_params *p, const void *d_in, vo
 tahq_status tahq_qnaive_decode(const tahq_qnaive_params *p, const void *d_packed, size_t packed_bytes, void *d_out,
                                void *d_ws, size_t ws_cap, tahq_stream stream);
 
+/*
+ * Self-test of the library's bounded device-side waits (the paper has no counterpart).  Launches a two-CTA
+ * kernel in which one CTA waits, as the offset look-back of encode/decode does, for a count that is never
+ * published.  The wait gives up after its fixed number of polls (about a second), the kernel returns, and
+ * the device status word at d_ws[0..4) reads TAHQ_DEV_TIMEOUT; the CUDA context stays usable.  d_ws: at
+ * least 32 KiB of device memory.
+ */
+tahq_status tahq_selftest_wait_timeout(void *d_ws, size_t ws_cap, tahq_stream stream);
+
 /* Static string for a status code. */
 const char *tahq_status_string(tahq_status s);
 

@@ -90,6 +90,7 @@ class QNaiveParams:
 EXPORTS = ["tahq_packed_bound", "tahq_packed_layout", "tahq_workspace_bound", "tahq_encode", "tahq_decode",
            "tahq_encode_noalloc",
            "tahq_qnaive_packed_bound", "tahq_qnaive_workspace_bound", "tahq_qnaive_encode", "tahq_qnaive_decode",
+           "tahq_selftest_wait_timeout",
            "tahq_status_string", "tahq_last_launch_count", "tahq_profile", "tahq_profile_read"]
 
 _lib = None
@@ -132,6 +133,8 @@ def lib() -> C.CDLL:
         L.tahq_qnaive_encode.restype = C.c_int
         L.tahq_qnaive_decode.argtypes = [qp, C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
         L.tahq_qnaive_decode.restype = C.c_int
+        L.tahq_selftest_wait_timeout.argtypes = [C.c_void_p, C.c_size_t, C.c_void_p]
+        L.tahq_selftest_wait_timeout.restype = C.c_int
         _lib = L
     return _lib
 
@@ -294,3 +297,8 @@ def qnaive_decode(p: QNaiveParams, packed: torch.Tensor, out: torch.Tensor | Non
     if rc:
         raise TahqError(rc)
     return out, ws
+
+
+def selftest_wait_timeout(ws: torch.Tensor) -> int:
+    """Run the bounded-wait self-test on `ws` (>= 32 KiB, device); returns the C status code."""
+    return int(lib().tahq_selftest_wait_timeout(ws.data_ptr(), ws.numel(), int(torch.cuda.current_stream(ws.device).cuda_stream)))

@@ -518,6 +518,20 @@ tahq_status tahq_qnaive_decode(const tahq_qnaive_params *p, const void *d_packed
   return cudaGetLastError() == cudaSuccess ? TAHQ_OK : TAHQ_ERR_CUDA;
 }
 
+tahq_status tahq_selftest_wait_timeout(void *d_ws, size_t ws_cap, tahq_stream stream) {
+  if (!d_ws) return TAHQ_ERR_INVALID_ARG;
+  if (ws_cap < 256 + 8ull * kMaxGrid) return TAHQ_ERR_BUFFER_TOO_SMALL;
+  if (!aligned16(d_ws)) return TAHQ_ERR_MISALIGNED;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  if (cudaMemsetAsync(d_ws, 0, 256 + 8ull * kMaxGrid, st) != cudaSuccess) return TAHQ_ERR_CUDA;
+  Args a;
+  std::memset(&a, 0, sizeof(a));
+  a.status = reinterpret_cast<uint32_t *>(d_ws);
+  a.flags = reinterpret_cast<unsigned long long *>(static_cast<uint8_t *>(d_ws) + 256);
+  wait_selftest_kernel<<<2, kThreads, 0, st>>>(a);
+  return cudaGetLastError() == cudaSuccess ? TAHQ_OK : TAHQ_ERR_CUDA;
+}
+
 const char *tahq_status_string(tahq_status s) {
   switch (s) {
     case TAHQ_OK: return "ok";

@@ -133,6 +133,14 @@ __device__ __forceinline__ uint64_t cta_exclusive_prefix(const Args &a, uint64_t
   return total;
 }
 
+// Self-test of the bounded waits: CTA 1 waits for a count that CTA 0 never publishes.  The wait gives
+// up after kSpinLimit polls, the status word gets TAHQ_DEV_TIMEOUT, and the kernel returns.
+__global__ void __launch_bounds__(kThreads) wait_selftest_kernel(const Args a) {
+  if (blockIdx.x == 0) return;
+  bool unused;
+  cta_exclusive_prefix(a, 1, false, unused);
+}
+
 // ------------------------------------------------------------------------------------------
 // Eq. 1-2: entropy score per tile, plus the per-group histogram of binned scores (Sec. 3.2)
 // ------------------------------------------------------------------------------------------

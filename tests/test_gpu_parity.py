@@ -269,3 +269,16 @@ def test_deterministic_and_stream_ordered():
     assert T.last_launch_count() > 0
     rel = ((y - x).double().pow(2).sum() / x.double().pow(2).sum()).item()
     assert rel < 0.05
+
+
+def test_bounded_wait_runs_out_and_reports():
+    """A device-side wait on a flag that nothing sets gives up after its fixed number of polls: the kernel
+    returns, the status word says TIMEOUT, and the context goes on working (an encode right after it)."""
+    ws = torch.empty(1 << 16, dtype=torch.uint8, device="cuda")
+    assert T.selftest_wait_timeout(ws) == 0
+    torch.cuda.synchronize()
+    assert T.device_status(ws) == 4                       # TAHQ_DEV_TIMEOUT
+    x = synth.make("c1_tiny", device="cuda")
+    p = T.params_for(x, group_tokens=64, tile=64, budget_millibits=3800)
+    packed, want, ws2 = check_encode(p, x)
+    check_decode(p, packed, want, ws2)
