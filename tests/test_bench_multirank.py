@@ -77,3 +77,65 @@ def test_shard_samples_partition(tokens, g, world):
         assert first == pos and count % (g or tokens) == 0
         pos += count
     assert pos == tokens
+
+
+class _OracleCodec:
+    """The boundary's codec interface, filled by the CPU oracle (the transport is what is under test here)."""
+
+    def __init__(self, kind, tokens, hidden):
+        self.kind = kind
+        if kind == "fw":
+            self.p = O.Params(tokens=tokens, hidden=hidden, dtype=0, group_tokens=64, tile=64, budget_millibits=3800)
+            self.nbytes = O.packed_bound(self.p)
+        else:
+            self.p = O.QNaiveParams(tokens=tokens, hidden=hidden, bits=6, prescale=1024.0)
+            self.nbytes = O.qnaive_packed_bound(self.p)
+
+    def encode(self, x):
+        f = O.encode if self.kind == "fw" else O.qnaive_encode
+        return torch.from_numpy(f(self.p, x.numpy()))
+
+    def decode(self, packed):
+        f = O.decode if self.kind == "fw" else O.qnaive_decode
+        return torch.from_numpy(f(self.p, packed.numpy()).reshape(self.p.tokens, self.p.hidden))
+
+
+def _boundary_worker(rank: int, world: int, port: int, out):
+    from paper_2506_01352_b200.boundary import Boundary
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        x = torch.from_numpy(synth.to_host_array(synth.make("c1_tiny", device="cpu")))
+        g = torch.from_numpy(synth.to_host_array(synth.make("c1_tiny", microbatch=1, device="cpu"))) * 1e-3
+        fw, bw = _OracleCodec("fw", 128, 256), _OracleCodec("bw", 128, 256)
+        b = Boundary(lower=0, upper=1, forward=fw, backward=bw,
+                     recv_buffer=lambda n: torch.empty(n, dtype=torch.uint8))
+        if rank == 0:
+            b.send_activations(x)                    # Algorithm 1 line 4
+            ghat = b.recv_gradient()                 # line 7
+            assert torch.equal(ghat, bw.decode(bw.encode(g)))
+        else:
+            xhat = b.recv_activations()              # line 5
+            assert torch.equal(xhat, fw.decode(fw.encode(x)))
+            assert float((xhat - x).abs().max()) < 0.6 * float(x.abs().max())
+            b.send_gradient(g)                       # line 6
+        out.put((rank, "ok"))
+    except Exception as e:
+        out.put((rank, repr(e)))
+    finally:
+        dist.destroy_process_group()
+
+
+def test_boundary_transport_two_ranks():
+    """Forward activations and backward gradients cross a two-stage boundary as fixed-size byte buffers."""
+    world = 2
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    port = _free_port()
+    procs = [ctx.Process(target=_boundary_worker, args=(r, world, port, q)) for r in range(world)]
+    for pr in procs:
+        pr.start()
+    res = dict(q.get(timeout=120) for _ in range(world))
+    for pr in procs:
+        pr.join(timeout=60)
+    assert res == {0: "ok", 1: "ok"}, res

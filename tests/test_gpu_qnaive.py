@@ -65,3 +65,20 @@ def test_refuses_a_foreign_buffer():
     out, ws = T.qnaive_decode(p2, packed, out=out)
     torch.cuda.synchronize()
     assert T.device_status(ws) & 1 and bool((out == 7.0).all())
+
+
+def test_boundary_codecs_on_one_device():
+    """The two codec objects a pipeline boundary uses (forward TAH-Quant, backward fixed point), round trip."""
+    from paper_2506_01352_b200.boundary import QNaiveCodec, TahqCodec
+    x = synth.make("c2_gpt2s", device="cuda")
+    fw = TahqCodec(x.shape[0], x.shape[1], x.dtype, x.device, group_tokens=1024, tile=64, budget_millibits=3800)
+    xh = fw.decode(fw.encode(x))
+    torch.cuda.synchronize()
+    assert fw.nbytes == fw.packed.numel() and xh.shape == x.shape
+    rel = float((xh - x).norm() / x.norm())
+    assert rel < 0.15
+    g = synth.make("c2_gpt2s", variant=1, device="cuda")
+    bw = QNaiveCodec(g.shape[0], g.shape[1], g.dtype, g.device, bits=6, prescale=1024.0)
+    gh = bw.decode(bw.encode(g))
+    torch.cuda.synchronize()
+    assert float((gh - g).abs().max()) <= float(g.abs().max()) / 31 / 2 * 1.001
