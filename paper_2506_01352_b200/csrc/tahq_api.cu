@@ -202,6 +202,36 @@ static unsigned persistent_grid(uint64_t n_chunks, const DevInfo &d, int occ) {
   return (unsigned)(n_chunks < cap ? n_chunks : cap);
 }
 
+// Tensor map of the input seen as [n_tiles rows x 128 bytes] with boxes of 32 rows and the 128-byte
+// swizzle, for the tiled TMA copies of the warp-streaming kernels.  The driver's encoder is looked up once
+// through the runtime (no link-time dependency on libcuda).  Returns false when TMA cannot be used here
+// (rows are not 128 bytes, too many rows for a 32-bit coordinate, or the encoder is unavailable).
+template <class C>
+static bool make_row_map(const void *in, uint64_t n_tiles, CUtensorMap *tm) {
+  std::memset(tm, 0, sizeof(*tm));
+  if (C::LPT != 1 || C::ROWB != 128 || n_tiles >= 0x7fffffe0ull) return false;
+  typedef CUresult (*encode_fn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+  static encode_fn enc = [] {
+    void *f = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+      f = nullptr;
+    return reinterpret_cast<encode_fn>(f);
+  }();
+  if (!enc) { cudaGetLastError(); return false; }
+  const cuuint64_t dims[2] = {(cuuint64_t)C::EPT, (cuuint64_t)n_tiles};
+  const cuuint64_t strides[1] = {128};
+  const cuuint32_t box[2] = {(cuuint32_t)C::EPT, 32};
+  const cuuint32_t estr[2] = {1, 1};
+  return enc(tm, C::BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2,
+             const_cast<void *>(in), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 // TAHQ_ENCODE_PATH=fused in the environment switches large-group encodes to the single cooperative kernel.
 // It is off by default: measured on B200 it never beat the three-kernel path (equal encode time on the
 // LLaMA-7B-shaped tensor, 7 % slower round trips because a cooperative launch does not overlap its
@@ -215,9 +245,12 @@ static bool fused_encode_wanted() {
 }
 
 template <class C, bool SR>
-static tahq_status encode_t(const Plan &pl, const Args &a, cudaStream_t st) {
+static tahq_status encode_t(const Plan &pl, const Args &a_in, cudaStream_t st) {
   DevInfo d;
   if (!dev_info(&d)) return TAHQ_ERR_CUDA;
+  Args a = a_in;
+  CUtensorMap tmap;
+  a.use_tma = make_row_map<C>(a.in, a.n_tiles, &tmap) ? 1u : 0u;
   const uint64_t n_chunks = (a.n_tiles + C::TPC - 1) / C::TPC;
   static std::atomic<int> occ_stats[64], occ_quant[64], sel_ready[64], occ_fused[64];
   if constexpr (C::LPT == 1) {
@@ -230,7 +263,7 @@ static tahq_status encode_t(const Plan &pl, const Args &a, cudaStream_t st) {
       if (occ) {
         const uint64_t n_units = (a.n_tiles + 31) / 32;
         const unsigned grid = persistent_grid((n_units + kWarps - 1) / kWarps, d, occ);
-        void *args[] = {const_cast<Args *>(&a)};
+        void *args[] = {&a, &tmap};
         cudaError_t e;
         {
           LaunchScope scope_("encode_fused", st);
@@ -246,13 +279,13 @@ static tahq_status encode_t(const Plan &pl, const Args &a, cudaStream_t st) {
   if (pl.mixed) {
     if constexpr (C::LPT == 1) {
       constexpr int NS = C::ROWB <= 128 ? 3 : 2;
-      const int smem = kWarps * NS * StreamCfg<C>::UNIT_BYTES;
+      const int smem = kWarps * NS * StreamCfg<C>::UNIT_BYTES + 256;   // ring slots, then the warps' mbarriers
       const int occ = prepare(stats_stream_kernel<C, NS>, smem, d, occ_stats);
       if (!occ) return TAHQ_ERR_CUDA;
       const uint64_t n_units = (a.n_tiles + 31) / 32;
       TAHQ_LAUNCH("stats", st,
                   stats_stream_kernel<C, NS><<<persistent_grid((n_units + kWarps - 1) / kWarps, d, occ), kThreads, smem,
-                                               st>>>(a));
+                                               st>>>(a, tmap));
     } else {
       constexpr int NS = Stages<C>::STATS;
       const int smem = NS * C::STAGE_BYTES;
@@ -276,7 +309,7 @@ static tahq_status encode_t(const Plan &pl, const Args &a, cudaStream_t st) {
     const uint64_t n_units = (a.n_tiles + 31) / 32;
     TAHQ_LAUNCH("quant_pack", st,
                 quant_pack_stream_kernel<C, NQ, SR><<<persistent_grid((n_units + kWarps - 1) / kWarps, d, occ), kThreads,
-                                                  smem, st>>>(a));
+                                                  smem, st>>>(a, tmap));
   } else {
     constexpr int NQ = Stages<C>::QUANT;
     const int smem = NQ * (C::STAGE_BYTES + C::TPC * 4);

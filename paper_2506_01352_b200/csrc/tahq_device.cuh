@@ -95,6 +95,16 @@ __device__ __forceinline__ bool mbar_wait(unsigned long long *bar, unsigned pari
   return false;
 }
 
+// Tiled TMA copy of a [rows x 128-byte] box of a two-dimensional tensor map into shared memory,
+// completing on an mbarrier.  x (the innermost coordinate) is always 0 here, so the 16-byte rule holds;
+// rows past the end of the tensor are filled with zeros by the hardware.
+__device__ __forceinline__ void tma_load_rows(void *dst, const void *tmap, int row0, unsigned long long *bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(smem_u32(dst)), "l"(tmap), "r"(0), "r"(row0), "r"(smem_u32(bar))
+      : "memory");
+}
+
 // Copy the rows of chunk `c` (tiles [c*TPC, (c+1)*TPC), clipped to n_tiles) into a swizzled stage.
 // Rows past the end of the tensor are zero-filled.
 template <class C>

@@ -36,6 +36,7 @@ struct Args {
   uint32_t direct;          // small groups: select_kernel ranks all scores of the group itself
   uint32_t exact_scores;    // stats_kernel writes exact scores (small groups, or a varsigma too large to screen)
   unsigned long long *flags;// [kMaxGrid] (zeroed per call) per-CTA published counts for the offset prefix
+  uint32_t use_tma;         // rows are 128 bytes and the tensor map is valid: units arrive by tiled TMA copies
   uint32_t *gbar;           // [2] (zeroed per call) arrival counters of the fused encode kernel's grid barriers
   uint32_t *status;         // device status word
   unsigned long long seed;  // stochastic rounding mode: the generator's key

@@ -15,6 +15,8 @@
 //     of work and no lane idles through the long path.
 #pragma once
 
+#include <cuda.h>   // CUtensorMap (type only; the driver entry point is looked up at run time)
+
 #include "tahq_kernels.cuh"
 
 namespace tahq {
@@ -27,7 +29,8 @@ struct StreamCfg {
   static_assert(C::LPT == 1, "one lane per tile");
   static constexpr int UNIT_BYTES = 32 * C::ROWB;   // 32 rows
   static constexpr int WORDS = C::ROWB / 4;         // 32-bit words of one row
-  static constexpr int smem_bytes(int nst) { return kWarps * (nst + 1) * UNIT_BYTES; }
+  // ring slots plus the stage of re-fetched rows, then the warps' mbarriers
+  static constexpr int smem_bytes(int nst) { return kWarps * (nst + 1) * UNIT_BYTES + 256; }
 };
 
 // cp.async of unit u (tiles 32u .. 32u+31) into a warp-private slot, rows swizzled as everywhere
@@ -53,6 +56,56 @@ __device__ __forceinline__ void warp_issue_unit(const uint8_t *in, uint64_t n_ti
     }
   }
 }
+
+// A warp's ring of unit slots.  Rows of 128 bytes arrive by one tiled TMA copy per unit, issued by
+// lane 0 and completing on the slot's mbarrier: the hardware's 128-byte swizzle is exactly the XOR
+// pattern of phys_chunk (slots are 1024-byte aligned), and rows past the end of the tensor come as
+// zeros.  Other row sizes use 16-byte cp.async per lane and commit groups.
+template <class C, int NST>
+struct UnitRing {
+  uint8_t *base;
+  unsigned long long *bar;   // [NST], this warp's
+  const void *tmap;          // nullptr: cp.async
+  uint32_t phases;           // bit s = parity slot s waits for next
+  int lane;
+  __device__ __forceinline__ void init(uint8_t *b, unsigned long long *br, const void *tm, int ln) {
+    base = b; bar = br; tmap = tm; phases = 0; lane = ln;
+    if (tmap) {
+      if (lane == 0) {
+#pragma unroll
+        for (int s = 0; s < NST; ++s) mbar_init(&bar[s], 1);
+        mbar_init_fence();
+      }
+      __syncwarp();
+    }
+  }
+  __device__ __forceinline__ uint8_t *slot(int s) const { return base + (size_t)s * StreamCfg<C>::UNIT_BYTES; }
+  // fill slot s with unit u; every lane is done reading the slot (the caller has synchronised the warp)
+  __device__ __forceinline__ void issue(const Args &a, uint64_t u, int s) {
+    if (tmap) {
+      if (lane == 0) {
+        fence_async_proxy();   // the lanes' reads of the slot are ordered before the asynchronous write
+        mbar_expect_tx(&bar[s], StreamCfg<C>::UNIT_BYTES);
+        tma_load_rows(slot(s), tmap, (int)(u * 32), &bar[s]);
+      }
+    } else {
+      warp_issue_unit<C>(a.in, a.n_tiles, u, slot(s), lane);
+    }
+  }
+  __device__ __forceinline__ void commit() const {   // one group per round, issued or not
+    if (!tmap) cp_async_commit();
+  }
+  // the unit issued into slot s has landed (call once per issue, in issue order)
+  __device__ __forceinline__ void wait(const Args &a, int s) {
+    if (tmap) {
+      if (!mbar_wait(&bar[s], (phases >> s) & 1u)) atomicOr(a.status, 4u /* TAHQ_DEV_TIMEOUT */);
+      phases ^= 1u << s;
+    } else {
+      cp_async_wait<NST - 1>();
+    }
+    __syncwarp();
+  }
+};
 
 // a row: shared memory <-> registers (raw words)
 template <class C>
@@ -105,10 +158,13 @@ __device__ __forceinline__ void words_minmax(const uint32_t (&w)[C::ROWB / 4], f
 // Eq. 1-2, warp-streaming: entropy score per tile, per-group histogram of binned scores (Sec. 3.2)
 // ------------------------------------------------------------------------------------------
 template <class C, int NST>
-__device__ __forceinline__ void stats_phase(const Args &a, uint8_t *smem, uint32_t *s_hist) {
+__device__ __forceinline__ void stats_phase(const Args &a, const void *tmap, uint8_t *smem, unsigned long long *bars,
+                                            uint32_t *s_hist) {
   using S = StreamCfg<C>;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  uint8_t *ring = smem + (size_t)warp * NST * S::UNIT_BYTES;
+  UnitRing<C, NST> ring;   // TMA needs 1024-byte aligned slots; otherwise the cp.async path does the same job
+  ring.init(smem + (size_t)warp * NST * S::UNIT_BYTES, bars + warp * NST,
+            (a.use_tma && (smem_u32(smem) & 1023u) == 0) ? tmap : nullptr, lane);
   const bool use_hist = !a.direct;
   const uint64_t n_units = (a.n_tiles + 31) / 32;
   const uint64_t u0 = n_units * blockIdx.x / gridDim.x, u1 = n_units * (blockIdx.x + 1ull) / gridDim.x;
@@ -125,23 +181,22 @@ __device__ __forceinline__ void stats_phase(const Args &a, uint8_t *smem, uint32
 #pragma unroll
     for (int s = 0; s < NST; ++s) {
       const uint64_t u = us + warp + (uint64_t)s * kWarps;
-      if (u < ue) warp_issue_unit<C>(a.in, a.n_tiles, u, ring + (size_t)s * S::UNIT_BYTES, lane);
-      cp_async_commit();
+      if (u < ue) ring.issue(a, u, s);
+      ring.commit();
     }
     __syncthreads();   // the histogram is clear
     int slot = 0;
     for (uint64_t u = us + warp; u < ue; u += kWarps) {
-      cp_async_wait<NST - 1>();
-      __syncwarp();
-      const uint8_t *stage = ring + (size_t)slot * S::UNIT_BYTES;
+      ring.wait(a, slot);
+      const uint8_t *stage = ring.slot(slot);
       // small groups are ranked on exact scores; large ones are screened first (see select_kernel)
       const float s = a.exact_scores ? tile_score<C>(stage, lane, a.eps_l1, a.eps_log)
                                      : tile_score_screen<C>(stage, lane, a.eps_l1);
       __syncwarp();
       {
         const uint64_t un = u + (uint64_t)NST * kWarps;
-        if (un < ue) warp_issue_unit<C>(a.in, a.n_tiles, un, ring + (size_t)slot * S::UNIT_BYTES, lane);
-        cp_async_commit();
+        if (un < ue) ring.issue(a, un, slot);
+        ring.commit();
       }
       slot = (slot + 1 == NST) ? 0 : slot + 1;
       const uint64_t tile = u * 32 + lane;
@@ -167,10 +222,12 @@ __device__ __forceinline__ void stats_phase(const Args &a, uint8_t *smem, uint32
 }
 
 template <class C, int NST>
-__global__ void __launch_bounds__(kThreads, 2) stats_stream_kernel(const Args a) {
-  extern __shared__ __align__(128) uint8_t smem[];
+__global__ void __launch_bounds__(kThreads, 2) stats_stream_kernel(const Args a, const __grid_constant__ CUtensorMap tmap) {
+  extern __shared__ __align__(1024) uint8_t smem_1k[];
+  uint8_t *smem = smem_1k;
   __shared__ uint32_t s_hist[kBins];   // this CTA's counts for the ranking group it is in
-  stats_phase<C, NST>(a, smem, s_hist);
+  stats_phase<C, NST>(a, &tmap, smem, reinterpret_cast<unsigned long long *>(smem + (size_t)kWarps * NST * StreamCfg<C>::UNIT_BYTES),
+                      s_hist);
 }
 
 // Sec. 3.3-3.4 for a row that is not transformed, straight from its raw words: zero-point and scale
@@ -318,8 +375,9 @@ __device__ __forceinline__ uint32_t scan_segment(const uint32_t *s_bm, uint32_t 
 constexpr int kQueueCap = 64;   // tile indices a warp can hold back (32 left over + 32 of one unit)
 
 template <class C, int NST, bool SR, bool COH>
-__device__ __forceinline__ void quant_phase(const Args &a, uint8_t *smem) {
+__device__ __forceinline__ void quant_phase(const Args &a, const void *tmap, uint8_t *smem) {
   using S = StreamCfg<C>;
+  unsigned long long *bars = reinterpret_cast<unsigned long long *>(smem + (size_t)kWarps * (NST + 1) * S::UNIT_BYTES);
   __shared__ uint32_t s_bm[kSegWords];    // bit-map words of the segment
   __shared__ uint32_t s_pre[kSegWords];   // higher-width tiles of the segment before each word
   __shared__ uint32_t s_wsum[kWarps];
@@ -327,8 +385,10 @@ __device__ __forceinline__ void quant_phase(const Args &a, uint8_t *smem) {
   __shared__ uint32_t s_qhib[kWarps][kQueueCap];    // held-back tile: higher-width tiles before it, from the CTA's first
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const unsigned lt = (1u << lane) - 1u;
-  uint8_t *ring = smem + (size_t)warp * (NST + 1) * S::UNIT_BYTES;
-  uint8_t *fstage = ring + (size_t)NST * S::UNIT_BYTES;   // rows fetched again for the flagged path
+  UnitRing<C, NST> ring;
+  ring.init(smem + (size_t)warp * (NST + 1) * S::UNIT_BYTES, bars + warp * NST,
+            (a.use_tma && (smem_u32(smem) & 1023u) == 0) ? tmap : nullptr, lane);
+  uint8_t *fstage = ring.slot(NST);   // rows fetched again for the flagged path (always by cp.async)
   uint32_t *sz32 = reinterpret_cast<uint32_t *>(a.packed + a.off_sz);
   uint8_t *pivot = a.packed + a.off_pivot;
   uint32_t *bitmap = reinterpret_cast<uint32_t *>(a.packed + a.off_bitmap);
@@ -343,8 +403,8 @@ __device__ __forceinline__ void quant_phase(const Args &a, uint8_t *smem) {
 #pragma unroll
     for (int s = 0; s < NST; ++s) {
       const uint64_t u = s0 + warp + (uint64_t)s * kWarps;
-      if (u < s1) warp_issue_unit<C>(a.in, a.n_tiles, u, ring + (size_t)s * S::UNIT_BYTES, lane);
-      cp_async_commit();
+      if (u < s1) ring.issue(a, u, s);
+      ring.commit();
     }
   };
   prime(u0, u0 + kSegWords < u1 ? u0 + kSegWords : u1);
@@ -456,19 +516,19 @@ __device__ __forceinline__ void quant_phase(const Args &a, uint8_t *smem) {
     // ---- the warp's units of this segment
     int slot = 0;
     for (uint64_t u = s0 + warp; u < s1; u += kWarps) {
-      cp_async_wait<NST - 1>();   // this unit has landed, and so have the rows fetched again one round ago
-      __syncwarp();
+      if (f_n && ring.tmap) cp_async_wait<0>();   // the rows fetched again one round ago (their own group here)
+      ring.wait(a, slot);                         // this unit has landed (cp.async: and so have those rows)
       if (f_n) run_flagged();
       if (qn >= 32u) gather(32u);
 
-      uint8_t *stage = ring + (size_t)slot * S::UNIT_BYTES;
+      uint8_t *stage = ring.slot(slot);
       uint32_t w[S::WORDS];
       row_load_words<C>(stage, lane, w);
       __syncwarp();
       {   // the slot is free again: fetch the unit that comes NST rounds later
         const uint64_t un = u + (uint64_t)NST * kWarps;
-        if (un < s1) warp_issue_unit<C>(a.in, a.n_tiles, un, stage, lane);
-        cp_async_commit();
+        if (un < s1) ring.issue(a, un, slot);
+        ring.commit();
       }
       slot = (slot + 1 == NST) ? 0 : slot + 1;
 
@@ -515,9 +575,10 @@ __device__ __forceinline__ void quant_phase(const Args &a, uint8_t *smem) {
 }
 
 template <class C, int NST, bool SR>
-__global__ void __launch_bounds__(kThreads, 2) quant_pack_stream_kernel(const Args a) {
-  extern __shared__ __align__(128) uint8_t smem[];
-  quant_phase<C, NST, SR, false>(a, smem);
+__global__ void __launch_bounds__(kThreads, 2) quant_pack_stream_kernel(const Args a, const __grid_constant__ CUtensorMap tmap) {
+  extern __shared__ __align__(1024) uint8_t smem_1k[];
+  uint8_t *smem = smem_1k;
+  quant_phase<C, NST, SR, false>(a, &tmap, smem);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -665,11 +726,14 @@ __device__ __forceinline__ void rank_group(const Args &a, uint64_t g, unsigned l
 }
 
 template <class C, bool SR>
-__global__ void __launch_bounds__(kThreads, 2) encode_fused_kernel(const Args a) {
+__global__ void __launch_bounds__(kThreads, 2) encode_fused_kernel(const Args a, const __grid_constant__ CUtensorMap tmap) {
   using S = StreamCfg<C>;
-  extern __shared__ __align__(128) uint8_t smem[];
-  // Eq. 1-2: two ring slots per warp, the CTA's histogram behind them
-  stats_phase<C, 2>(a, smem, reinterpret_cast<uint32_t *>(smem + (size_t)kWarps * 2 * S::UNIT_BYTES));
+  extern __shared__ __align__(1024) uint8_t smem_1k[];
+  uint8_t *smem = smem_1k;
+  // Eq. 1-2: two ring slots per warp, the CTA's histogram behind them; mbarriers at the very end
+  stats_phase<C, 2>(a, &tmap, smem,
+                    reinterpret_cast<unsigned long long *>(smem + (size_t)kWarps * 3 * S::UNIT_BYTES + 128),
+                    reinterpret_cast<uint32_t *>(smem + (size_t)kWarps * 2 * S::UNIT_BYTES));
   grid_barrier(a, 0);   // every histogram is complete
   const uint64_t n_units = (a.n_tiles + 31) / 32;
   const uint64_t u0 = n_units * blockIdx.x / gridDim.x, u1 = n_units * (blockIdx.x + 1ull) / gridDim.x;
@@ -686,7 +750,7 @@ __global__ void __launch_bounds__(kThreads, 2) encode_fused_kernel(const Args a)
     const uint64_t g0 = t0 / a.tiles_per_group, g1 = (t1 - 1) / a.tiles_per_group;
     for (uint64_t g = g0; g <= g1; ++g) rank_group(a, g, reinterpret_cast<unsigned long long *>(smem));
   }
-  quant_phase<C, 2, SR, true>(a, smem);
+  quant_phase<C, 2, SR, true>(a, &tmap, smem);
 }
 
 // ------------------------------------------------------------------------------------------
