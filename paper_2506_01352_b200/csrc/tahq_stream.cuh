@@ -513,9 +513,15 @@ __device__ __forceinline__ void quant_phase(const Args &a, const void *tmap, uin
     }
     __syncthreads();
 
-    // ---- the warp's units of this segment
+    // ---- the warp's units of this segment; inside the loop everything is relative to the CTA's first
+    // tile and first payload byte, in 32-bit arithmetic
     int slot = 0;
-    for (uint64_t u = s0 + warp; u < s1; u += kWarps) {
+    uint8_t *const pay_cta = payload + (uint64_t)(C::G / 8) * ((uint64_t)a.lo * tile_cta + base_hi);
+    uint32_t *const sz_cta = sz32 + tile_cta;
+    uint8_t *const pv_cta = pivot + tile_cta;
+    const uint32_t n_rel = a.n_tiles - tile_cta < 0xffffffffull ? (uint32_t)(a.n_tiles - tile_cta) : 0xffffffffu;
+    const uint32_t su1 = (uint32_t)(s1 - s0), seg_rel = (uint32_t)(s0 - u0) * 32u;
+    for (uint32_t su = warp; su < su1; su += kWarps) {   // su = unit index inside the segment
       if (f_n && ring.tmap) cp_async_wait<0>();   // the rows fetched again one round ago (their own group here)
       ring.wait(a, slot);                         // this unit has landed (cp.async: and so have those rows)
       if (f_n) run_flagged();
@@ -526,17 +532,17 @@ __device__ __forceinline__ void quant_phase(const Args &a, const void *tmap, uin
       row_load_words<C>(stage, lane, w);
       __syncwarp();
       {   // the slot is free again: fetch the unit that comes NST rounds later
-        const uint64_t un = u + (uint64_t)NST * kWarps;
-        if (un < s1) ring.issue(a, un, slot);
+        const uint32_t sn = su + (uint32_t)NST * kWarps;
+        if (sn < su1) ring.issue(a, s0 + sn, slot);
         ring.commit();
       }
       slot = (slot + 1 == NST) ? 0 : slot + 1;
 
-      const uint32_t word = s_bm[u - s0];
+      const uint32_t word = s_bm[su];
       const uint32_t hi = (word >> lane) & 1u;
-      const uint64_t tile = u * 32 + lane;
-      const bool live = tile < a.n_tiles;
-      const uint32_t hib = s_pre[u - s0] + (uint32_t)__popc(word & lt);
+      const uint32_t trel = seg_rel + su * 32u + lane;   // tile - first tile of the CTA
+      const bool live = trel < n_rel;
+      const uint32_t hib = s_pre[su] + (uint32_t)__popc(word & lt);
 
       // Eq. 3, first look: the second-largest magnitude is at least the smaller of |min| and |max| (they
       // sit at different positions, or every element is equal), so a tile whose largest magnitude does
@@ -548,15 +554,15 @@ __device__ __forceinline__ void quant_phase(const Args &a, const void *tmap, uin
       const unsigned held = __ballot_sync(kFull, maybe);
       if (maybe) {
         const uint32_t e = (qhead + qn + (uint32_t)__popc(held & lt)) & (kQueueCap - 1);
-        s_qtile[warp][e] = (uint32_t)((tile - tile_cta) << 1) | hi;
+        s_qtile[warp][e] = (trel << 1) | hi;
         s_qhib[warp][e] = hib;
       }
       qn += (uint32_t)__popc(held);
       if (live && !maybe) {
-        const uint64_t off = (uint64_t)(C::G / 8) * ((uint64_t)a.lo * tile + base_hi + hib);
-        sz32[tile] = encode_plain_words<C, SR>(w, mn, mx, a.lo + hi, narrow, reinterpret_cast<uint32_t *>(payload + off),
-                                               a.seed, tile * (unsigned long long)C::G);
-        pivot[tile] = 0;
+        const uint32_t off = (uint32_t)(C::G / 8) * (a.lo * trel + hib);
+        sz_cta[trel] = encode_plain_words<C, SR>(w, mn, mx, a.lo + hi, narrow, reinterpret_cast<uint32_t *>(pay_cta + off),
+                                                 a.seed, (tile_cta + trel) * (unsigned long long)C::G);
+        pv_cta[trel] = 0;
       }
       __syncwarp();
     }
