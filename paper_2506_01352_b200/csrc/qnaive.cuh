@@ -10,6 +10,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <type_traits>
+
 namespace tahq {
 
 struct QArgs {
@@ -89,41 +91,75 @@ __global__ void __launch_bounds__(kQThreads, 2) qnaive_encode_kernel(const QArgs
   // pieces a lane's b bytes are stored in: the largest power of two dividing b, at most 16
   const uint32_t gsz = (b & (0u - b)) > 16u ? 16u : (b & (0u - b));
 
-  // one group of eight elements -> the lane's b bytes of codes at dst
-  auto emit = [&](const float (&v)[8], float inv, uint8_t *dst) {
-    unsigned long long lo = 0, hi = 0;   // b bytes as a 128-bit little-endian value
+  // one group of eight elements -> the lane's b bytes of codes at dst.  B > 0: the width as a compile-time
+  // constant (all shifts static, 32-bit words); B == 0: any width, 128-bit value built with run-time shifts.
+  auto emit_w = [&](auto Bc, const float (&v)[8], float inv, uint8_t *dst) {
+    constexpr int B = decltype(Bc)::value;
+    int q[8];
 #pragma unroll
     for (int k = 0; k < 8; ++k) {
       const float y = a.prescale * v[k];
       const float t = __fmaf_rn(y, inv, kQMagic);   // one rounding, ties to even
-      int q = (int)(__float_as_uint(t) - 0x4B400000u);
-      q = min(max(q, -Lq), Lq);
-      const unsigned long long code = (unsigned long long)(uint32_t)(q + Lq);
-      const uint32_t pos = (uint32_t)k * b;
-      if (pos < 64) {
-        lo |= code << pos;
-        if (pos + b > 64) hi |= code >> (64 - pos);
+      q[k] = min(max((int)(__float_as_uint(t) - 0x4B400000u), -Lq), Lq) + Lq;
+    }
+    if constexpr (B > 0) {
+      uint32_t w[B / 4 + 1];
+#pragma unroll
+      for (int j = 0; j < B / 4 + 1; ++j) w[j] = 0;
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        constexpr int dummy = 0; (void)dummy;
+        const int pos = k * B, wi = pos >> 5, sh = pos & 31;
+        w[wi] |= (uint32_t)q[k] << sh;
+        if (sh + B > 32) w[wi + 1] |= (uint32_t)q[k] >> (32 - sh);
+      }
+      if constexpr (B == 16) *reinterpret_cast<uint4 *>(dst) = make_uint4(w[0], w[1], w[2], w[3]);
+      else if constexpr (B == 8) *reinterpret_cast<uint2 *>(dst) = make_uint2(w[0], w[1]);
+      else if constexpr (B % 4 == 0) {
+#pragma unroll
+        for (int j = 0; j < B / 4; ++j) reinterpret_cast<uint32_t *>(dst)[j] = w[j];
+      } else {   // even widths: 16-bit pieces
+#pragma unroll
+        for (int j = 0; j < B / 2; ++j) reinterpret_cast<uint16_t *>(dst)[j] = (uint16_t)(w[j >> 1] >> (16 * (j & 1)));
+      }
+    } else {
+      unsigned long long lo = 0, hi = 0;
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        const unsigned long long code = (unsigned long long)(uint32_t)q[k];
+        const uint32_t pos = (uint32_t)k * b;
+        if (pos < 64) {
+          lo |= code << pos;
+          if (pos + b > 64) hi |= code >> (64 - pos);
+        } else {
+          hi |= code << (pos - 64);
+        }
+      }
+      if (gsz == 4) {
+#pragma unroll
+        for (int j = 0; j < 3; ++j)
+          if ((uint32_t)(4 * j) < b) reinterpret_cast<uint32_t *>(dst)[j] = (uint32_t)(j < 2 ? lo >> (32 * j) : hi);
+      } else if (gsz == 2) {
+#pragma unroll
+        for (int j = 0; j < 7; ++j)
+          if ((uint32_t)(2 * j) < b)
+            reinterpret_cast<uint16_t *>(dst)[j] = (uint16_t)(j < 4 ? lo >> (16 * j) : hi >> (16 * (j - 4)));
       } else {
-        hi |= code << (pos - 64);
+#pragma unroll
+        for (int j = 0; j < 15; ++j)
+          if ((uint32_t)j < b) dst[j] = (uint8_t)(j < 8 ? lo >> (8 * j) : hi >> (8 * (j - 8)));
       }
     }
-    if (gsz == 16) {
-      *reinterpret_cast<uint4 *>(dst) = make_uint4((uint32_t)lo, (uint32_t)(lo >> 32), (uint32_t)hi, (uint32_t)(hi >> 32));
-    } else if (gsz == 8) {
-      *reinterpret_cast<unsigned long long *>(dst) = lo;
-    } else if (gsz == 4) {
-#pragma unroll
-      for (int j = 0; j < 3; ++j)
-        if ((uint32_t)(4 * j) < b) reinterpret_cast<uint32_t *>(dst)[j] = (uint32_t)(j < 2 ? lo >> (32 * j) : hi);
-    } else if (gsz == 2) {
-#pragma unroll
-      for (int j = 0; j < 7; ++j)
-        if ((uint32_t)(2 * j) < b)
-          reinterpret_cast<uint16_t *>(dst)[j] = (uint16_t)(j < 4 ? lo >> (16 * j) : hi >> (16 * (j - 4)));
-    } else {
-#pragma unroll
-      for (int j = 0; j < 15; ++j)
-        if ((uint32_t)j < b) dst[j] = (uint8_t)(j < 8 ? lo >> (8 * j) : hi >> (8 * (j - 8)));
+  };
+  auto emit = [&](const float (&v)[8], float inv, uint8_t *dst) {
+    switch (b) {   // uniform: the widths the paper uses (6, 8, 10) and their neighbours get static code
+      case 4: emit_w(std::integral_constant<int, 4>{}, v, inv, dst); break;
+      case 6: emit_w(std::integral_constant<int, 6>{}, v, inv, dst); break;
+      case 8: emit_w(std::integral_constant<int, 8>{}, v, inv, dst); break;
+      case 10: emit_w(std::integral_constant<int, 10>{}, v, inv, dst); break;
+      case 12: emit_w(std::integral_constant<int, 12>{}, v, inv, dst); break;
+      case 16: emit_w(std::integral_constant<int, 16>{}, v, inv, dst); break;
+      default: emit_w(std::integral_constant<int, 0>{}, v, inv, dst); break;
     }
   };
   constexpr int kHeld = BF16 ? 16 : 8;   // groups of eight elements a lane keeps in registers (64 registers)
@@ -236,31 +272,66 @@ __global__ void __launch_bounds__(kQThreads) qnaive_decode_kernel(const QArgs a)
     uint8_t *orow = a.out + r * (uint64_t)C * ESZ;
 #pragma unroll 4
     for (uint32_t k0 = lane * 8; k0 < C; k0 += 256) {
-      // the lane's b bytes start at byte o of the row; fetch the five aligned words that cover them
-      const uint32_t o = (k0 >> 3) * b, o4 = o & ~3u, sh = (o & 3u) * 8u;
-      uint32_t w[5];
+      // the lane's b bytes start at byte o of the row
+      const uint32_t o = (k0 >> 3) * b;
+      unsigned long long lo, hi = 0;
+      if (b == 8) {
+        lo = __ldg(reinterpret_cast<const unsigned long long *>(irow + o));
+      } else if (b == 16) {
+        const uint4 v = __ldg(reinterpret_cast<const uint4 *>(irow + o));
+        lo = (unsigned long long)v.x | ((unsigned long long)v.y << 32);
+        hi = (unsigned long long)v.z | ((unsigned long long)v.w << 32);
+      } else {   // the aligned words that cover them (four do unless the bytes start off a word boundary)
+        const uint32_t o4 = o & ~3u, sh = (o & 3u) * 8u;
+        uint32_t w[5];
 #pragma unroll
-      for (int j = 0; j < 5; ++j)
-        w[j] = (o4 + 4u * j < (uint32_t)a.row_bytes) ? __ldg(reinterpret_cast<const uint32_t *>(irow + o4) + j) : 0u;
-      uint32_t x[4];
+        for (int j = 0; j < 5; ++j)
+          w[j] = (o4 + 4u * j < (uint32_t)a.row_bytes && (j < 4 || sh)) ? __ldg(reinterpret_cast<const uint32_t *>(irow + o4) + j) : 0u;
+        uint32_t x[4];
 #pragma unroll
-      for (int j = 0; j < 4; ++j) x[j] = __funnelshift_r(w[j], w[j + 1], sh);
-      const unsigned long long lo = (unsigned long long)x[0] | ((unsigned long long)x[1] << 32);
-      const unsigned long long hi = (unsigned long long)x[2] | ((unsigned long long)x[3] << 32);
+        for (int j = 0; j < 4; ++j) x[j] = __funnelshift_r(w[j], w[j + 1], sh);
+        lo = (unsigned long long)x[0] | ((unsigned long long)x[1] << 32);
+        hi = (unsigned long long)x[2] | ((unsigned long long)x[3] << 32);
+      }
       float g[8];
+      auto codes = [&](auto Bc) {
+        constexpr int B = decltype(Bc)::value;
 #pragma unroll
-      for (int k = 0; k < 8; ++k) {
-        const uint32_t pos = (uint32_t)k * b;
-        unsigned long long c;
-        if (pos < 64) {
-          c = lo >> pos;
-          if (pos + b > 64) c |= hi << (64 - pos);
-        } else {
-          c = hi >> (pos - 64);
+        for (int k = 0; k < 8; ++k) {
+          unsigned long long c;
+          if constexpr (B > 0) {
+            constexpr int pos = 0; (void)pos;
+            const int p0 = k * B;
+            if (p0 < 64) {
+              c = lo >> p0;
+              if (p0 + B > 64) c |= hi << (64 - p0);
+            } else {
+              c = hi >> (p0 - 64);
+            }
+            c &= (1ull << B) - 1ull;
+          } else {
+            const uint32_t p0 = (uint32_t)k * b;
+            if (p0 < 64) {
+              c = lo >> p0;
+              if (p0 + b > 64) c |= hi << (64 - p0);
+            } else {
+              c = hi >> (p0 - 64);
+            }
+            c &= mask;
+          }
+          const int q = (int)(uint32_t)c - Lq;
+          const float t = __fmul_rn((float)q, s);
+          g[k] = pow2 ? __fmul_rn(t, rc) : __fdiv_rn(t, a.prescale);
         }
-        const int q = (int)(uint32_t)(c & mask) - Lq;
-        const float t = __fmul_rn((float)q, s);
-        g[k] = pow2 ? __fmul_rn(t, rc) : __fdiv_rn(t, a.prescale);
+      };
+      switch (b) {
+        case 4: codes(std::integral_constant<int, 4>{}); break;
+        case 6: codes(std::integral_constant<int, 6>{}); break;
+        case 8: codes(std::integral_constant<int, 8>{}); break;
+        case 10: codes(std::integral_constant<int, 10>{}); break;
+        case 12: codes(std::integral_constant<int, 12>{}); break;
+        case 16: codes(std::integral_constant<int, 16>{}); break;
+        default: codes(std::integral_constant<int, 0>{}); break;
       }
       if constexpr (BF16) {
         uint32_t u[4];
