@@ -3,8 +3,10 @@
 // Work decomposition: ONE THREAD OWNS ONE TILE (quantisation group, Sec. 3.1) -- or half of a
 // 128-wide tile -- and keeps its elements in registers, so that the Hadamard butterfly (Eq. 4),
 // the reductions of Eq. 1-3 and the bit packing need no cross-lane traffic.  Tiles reach the
-// thread through shared memory: a CTA copies 256 thread-rows with 16-byte cp.async into an
-// XOR-swizzled stage from which every thread reads its own row with conflict-free 128-bit loads.
+// thread through shared memory: rows are copied (16-byte cp.async, or tiled TMA with the 128-byte
+// swizzle) into an XOR-swizzled stage from which every thread reads its own row with conflict-free
+// 128-bit loads.  tahq_stream.cuh builds per-warp stages of 32 rows from these blocks,
+// tahq_kernels.cuh per-CTA stages of 256 thread-rows (128-wide tiles, two lanes per tile).
 #pragma once
 
 #include <cuda_bf16.h>

@@ -1,14 +1,14 @@
-// Kernels of the TAH-Quant boundary codec (sm_100a).  See tahq_device.cuh for the work decomposition.
+// Kernels of the TAH-Quant boundary codec (sm_100a) that work CTA-wide.  See tahq_device.cuh for the
+// work decomposition and tahq_stream.cuh for the warp-streaming kernels of tiles owned by one lane.
 //
-//   encode:  stats_kernel        Eq. 1-2   tile -> entropy score, per-group histogram of binned scores
-//                                          (skipped for integer budgets)
-//            select_kernel       Sec. 3.2  threshold bin, its candidates, exact k_hi-th (score, index) key
-//            quant_pack_stream_kernel (tahq_stream.cuh; tiles owned by one lane, G = 32, 64)
-//            quant_pack_kernel        (tiles owned by two lanes, G = 128)
-//                                Eq. 3-4, Sec. 3.2-3.4  bit map + offsets (prefix over CTAs), pivot test,
-//                                          swap + Hadamard, quantise, pack
-//   decode:  decode_kernel       Sec. 3.3, Alg. 1 l.5  header check, offsets from the bit map, unpack,
-//                                          z + q*s, inverse transform, store
+//   select_kernel       Sec. 3.2  threshold bin, its candidates, exact k_hi-th (score, index) key
+//   tiles owned by two lanes (G = 128), 256 thread-rows per CTA and stage:
+//   stats_kernel        Eq. 1-2   tile -> entropy score, per-group histogram of binned scores
+//                                 (skipped for integer budgets)
+//   quant_pack_kernel   Eq. 3-4, Sec. 3.2-3.4  bit map + offsets (prefix over CTAs), pivot test,
+//                                 swap + Hadamard, quantise, pack
+//   decode_kernel       Sec. 3.3, Alg. 1 l.5  header check, offsets from the bit map, unpack,
+//                                 z + q*s, inverse transform, store
 #pragma once
 
 #include "tahq_device.cuh"

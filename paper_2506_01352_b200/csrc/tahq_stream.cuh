@@ -1,18 +1,22 @@
-// Warp-streaming encode kernel of the TAH-Quant boundary codec (sm_100a), for tiles owned by one lane
-// (G = 32, 64).
+// Warp-streaming kernels of the TAH-Quant boundary codec (sm_100a), for tiles owned by one lane
+// (G = 32, 64): scores (Eq. 1-2), quantise + pack (Eq. 3-4, Sec. 3.2-3.4), decode (Sec. 3.3), and the
+// optional single-launch encode that runs the first two with grid-wide barriers in between.
 //
 // Every warp is an independent worker: it streams units of 32 consecutive tiles (one bit-map word)
-// through a private cp.async ring in shared memory, one lane per tile, and never meets a CTA-wide
-// barrier after the prologue.  Two things make that possible.
-//   * Sec. 3.2 / 3.4: the widths are known before the kernel starts (scores and thresholds are in
-//     memory), so the prologue turns the CTA's slice of scores into bit-map words, their running
+// through a private ring of slots in shared memory, one lane per tile, and never meets a CTA-wide
+// barrier after the prologue.  Rows of 128 bytes arrive by one tiled TMA copy per unit on the warp's
+// own mbarriers, other row sizes by 16-byte cp.async.  Two things make the independence possible.
+//   * Sec. 3.2 / 3.4: the widths are known before quantise + pack starts (scores and thresholds are
+//     in memory), so the prologue turns the CTA's slice of scores into bit-map words, their running
 //     population count, and (one look-back over the CTAs) the byte offset of every tile.
 //   * Eq. 3-4: tiles that pass the pivot test cost about three times as much as the others.  A lane
 //     handles an unflagged tile on the spot; tiles that may be flagged are only noted in a queue of
 //     tile indices private to the warp.  When 32 are queued, their rows are fetched again (from L2,
 //     where they were a moment ago) into a 32-row stage of the warp, and one iteration later the whole
-//     warp runs the flagged path on them, one lane per row.  All warps therefore do the same amount
-//     of work and no lane idles through the long path.
+//     warp runs the flagged path on them, one lane per row, in a routine that is not inlined (the
+//     hot loop stays small enough for the instruction cache).  All warps therefore do the same
+//     amount of work and no lane idles through the long path.  Decode holds transformed tiles back
+//     in the same way.
 #pragma once
 
 #include <cuda.h>   // CUtensorMap (type only; the driver entry point is looked up at run time)
