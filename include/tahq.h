@@ -151,7 +151,7 @@ tahq_status tahq_decode(const tahq_params *p, const void *d_packed, size_t packe
  *
  * Limits and rules
  *   - Accepts exactly the configurations with tahq_workspace_bound(p) <= TAHQ_NOALLOC_SCRATCH_BYTES
- *     (e.g. 8192 x 4096 elements at tile 64 needs 3.2 MB); anything larger returns
+ *     (e.g. 8192 x 4096 elements at tile 64 needs 3.3 MB); anything larger returns
  *     TAHQ_ERR_TOO_LARGE and enqueues nothing.
  *   - The first call on each device looks up the device address of the built-in buffer (a host-side
  *     set-up step, done once per device with that device current).  Make that first call before any

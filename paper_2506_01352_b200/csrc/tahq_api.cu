@@ -50,6 +50,19 @@ struct Plan {
 
 static uint64_t up(uint64_t x, uint64_t a) { return (x + a - 1) / a * a; }
 
+// TAHQ_ENCODE_PATH=fused in the environment switches large-group encodes to the single cooperative kernel.
+// It is off by default: measured on B200 it never beat the three-kernel path (equal encode time on the
+// LLaMA-7B-shaped tensor, 7 % slower round trips because a cooperative launch does not overlap its
+// neighbours' launch latency; 7-13 % slower on 320 MiB and 1 GiB tensors).
+static bool fused_encode_wanted() {
+  static const bool v = [] {
+    const char *e = std::getenv("TAHQ_ENCODE_PATH");
+    return e && std::strcmp(e, "fused") == 0;
+  }();
+  return v;
+}
+
+
 static tahq_status make_plan(const tahq_params *p, Plan *pl) {
   if (!p || p->struct_size != sizeof(tahq_params)) return TAHQ_ERR_INVALID_ARG;
   const uint32_t G = p->tile;
@@ -89,8 +102,10 @@ static tahq_status make_plan(const tahq_params *p, Plan *pl) {
   pl->cand_cap = 0;
   if (pl->mixed && !pl->direct) {
     pl->cpg = (uint32_t)((L.tiles_per_group + kSelSlice - 1) / kSelSlice);
-    // every tile of a group can end up a candidate (all scores equal): the list holds them all
-    pl->cand_cap = (uint32_t)(L.tiles_per_group < 0xffffffffull ? L.tiles_per_group : 0xffffffffull);
+    // select_kernel copes with more candidates than the list holds; the single-launch encode does not, so
+    // there the list holds a whole group (every tile is a candidate when all scores are equal)
+    const uint64_t cap = fused_encode_wanted() ? 0xffffffffull : 32768ull;
+    pl->cand_cap = (uint32_t)(L.tiles_per_group < cap ? L.tiles_per_group : cap);
   }
   const bool hist = pl->mixed && !pl->direct;
   uint64_t o = 256;                                         // status word and friends
@@ -230,18 +245,6 @@ static bool make_row_map(const void *in, uint64_t n_tiles, CUtensorMap *tm) {
              const_cast<void *>(in), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
-// TAHQ_ENCODE_PATH=fused in the environment switches large-group encodes to the single cooperative kernel.
-// It is off by default: measured on B200 it never beat the three-kernel path (equal encode time on the
-// LLaMA-7B-shaped tensor, 7 % slower round trips because a cooperative launch does not overlap its
-// neighbours' launch latency; 7-13 % slower on 320 MiB and 1 GiB tensors).
-static bool fused_encode_wanted() {
-  static const bool v = [] {
-    const char *e = std::getenv("TAHQ_ENCODE_PATH");
-    return e && std::strcmp(e, "fused") == 0;
-  }();
-  return v;
 }
 
 template <class C, bool SR>
