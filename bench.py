@@ -47,6 +47,7 @@ def parse_args():
     ap.add_argument("--variant", type=int, default=0)
     ap.add_argument("--budget", type=int, default=3800)
     ap.add_argument("--tile", type=int, default=64)
+    ap.add_argument("--sets", type=int, default=4, help="distinct input/packed/output buffer sets rotated through")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     return ap.parse_args()
 
@@ -178,7 +179,7 @@ def main():
     T.lib()
 
     w = synth.WORKLOADS[args.workload]
-    n_sets = 4
+    n_sets = max(1, args.sets)
     # every rank encodes/decodes its own boundary tensors (one per pipeline-stage boundary): no collective
     xs = [synth.make(args.workload, variant=args.variant, microbatch=mb, device=dev)
           for mb in shard.rank_microbatches(rank, n_sets)]
