@@ -38,6 +38,7 @@ class _Params(C.Structure):
         ("eps_ratio", C.c_float),
         ("rounding", C.c_uint32),
         ("seed", C.c_uint64),
+        ("alloc_tile", C.c_uint32),
     ]
 
 
@@ -99,11 +100,12 @@ class Params:
     eps_ratio: float = 1e-8
     rounding: int = 0
     seed: int = 0
+    alloc_tile: int = 0          # A of Sec. 3.2 (0 = the quantisation tile)
 
     def c(self) -> _Params:
         return _Params(self.dtype, self.tokens, self.hidden, self.group_tokens, self.tile,
                        self.budget_millibits, self.tau, self.eps_l1, self.eps_log, self.eps_ratio,
-                       self.rounding, self.seed)
+                       self.rounding, self.seed, self.alloc_tile)
 
 
 def build(force: bool = False) -> str:

@@ -106,12 +106,17 @@ int tahqo_layout_of(const tahqo_params *p, tahqo_layout *L) {
   uint32_t beta = p->budget_millibits;
   if (beta < 2000 || beta > 8000) return 1;
   uint32_t lo = beta / 1000, f = beta % 1000;
-  uint64_t M = p->hidden / G;                                 /* tiles per token (Sec. 3.2, A = G) */
+  uint64_t M = p->hidden / G;                                 /* quantisation tiles per token */
+  uint32_t A = p->alloc_tile ? p->alloc_tile : G;             /* allocation-tile width (Sec. 3.2) */
+  if (A % G || A > p->hidden || p->hidden % A) return 1;
+  uint64_t m = A / G;                                         /* quantisation tiles per allocation tile */
   L->n_tiles = p->tokens * M;
-  L->tiles_per_group = S * M;                                 /* "the SM allocation tiles of every sample" */
+  L->tiles_per_group = S * M;
   L->n_groups = p->tokens / S;
-  /* top-p% with p = f/10 percent: never more than the budget allows */
-  L->k_hi = (L->tiles_per_group * (uint64_t)f) / 1000u;
+  /* "the SM allocation tiles of every sample" (M = C/A here): top-p% of them, p = f/10 percent, never
+   * more than the budget allows; every quantisation tile inside a chosen allocation tile gets hi */
+  uint64_t alloc_per_group = S * (p->hidden / A);
+  L->k_hi = ((alloc_per_group * (uint64_t)f) / 1000u) * m;
   L->lo_bits = lo;
   L->hi_bits = f ? lo + 1 : lo;
   L->payload_bytes = L->n_groups * (uint64_t)(G / 8) * (L->tiles_per_group * lo + L->k_hi);
@@ -153,21 +158,26 @@ static void write_header(const tahqo_params *p, const tahqo_layout *L, uint8_t *
   put64(h + 64, L->n_tiles);
   put64(h + 72, L->payload_bytes);
   put64(h + 80, L->total_bytes);
+  put32(h + 88, (p->alloc_tile && p->alloc_tile != p->tile) ? p->alloc_tile : 0u);   /* 0: A = G */
 }
 
 /* ------------------------------------------------------------------ */
 /* Steps                                                               */
 /* ------------------------------------------------------------------ */
 
-/* Fixed pairwise summation tree over n = 2^m values: neighbours first, then
- * neighbours of the partial sums, ...  Fixing the order makes every score a
- * single well-defined binary32 number (the paper does not give an order). */
+/* Fixed pairwise summation tree over n values: neighbours first, then
+ * neighbours of the partial sums, ... (a partial sum without a neighbour
+ * waits for the next level).  Fixing the order makes every score a single
+ * well-defined binary32 number (the paper does not give an order). */
 float tahqo_treesum(const float *x, uint32_t n) {
-  float t[128];
+  float small[128] = {0};
+  float *t = n <= 128 ? small : (float *)malloc((size_t)n * sizeof(float));
   for (uint32_t i = 0; i < n; i++) t[i] = x[i];
   for (uint32_t h = 1; h < n; h *= 2)
     for (uint32_t i = 0; i + h < n; i += 2 * h) t[i] = t[i] + t[i + h];
-  return t[0];
+  float r = t[0];
+  if (t != small) free(t);
+  return r;
 }
 
 /* log2 of a positive normal binary32 number: exponent + u*Q(u), u = mantissa-1
@@ -198,7 +208,11 @@ void tahqo_lg2_array(const float *x, float *y, size_t n) {
  * spread energy and low for a sharp outlier, which is Shannon's sign; the
  * score is therefore -sum p log2(p + varsigma). */
 float tahqo_score(const float *tile, uint32_t G, float eps_l1, float eps_log) {
-  float a[128] = {0}, term[128] = {0};
+  /* G is the width of the allocation tile the score is taken over (A of Sec. 3.2; = the quantisation
+   * tile by default) */
+  float sa[128] = {0}, st[128] = {0};
+  float *a = G <= 128 ? sa : (float *)malloc((size_t)G * sizeof(float));
+  float *term = G <= 128 ? st : (float *)malloc((size_t)G * sizeof(float));
   for (uint32_t k = 0; k < G; k++) a[k] = fabsf(tile[k]);
   float L1 = tahqo_treesum(a, G);
   float inv = 1.0f / (L1 + eps_l1);
@@ -206,7 +220,9 @@ float tahqo_score(const float *tile, uint32_t G, float eps_l1, float eps_log) {
     float p = a[k] * inv;                     /* Eq. 1 */
     term[k] = p * oracle_lg2(p + eps_log);    /* summand of Eq. 2 */
   }
-  return 0.0f - tahqo_treesum(term, G);
+  float r = 0.0f - tahqo_treesum(term, G);
+  if (a != sa) { free(a); free(term); }
+  return r;
 }
 
 /* Sec. 3.2 "Top-p% tile selection" inside one ranking group: sort the tiles by
@@ -378,19 +394,27 @@ int tahqo_encode(const tahqo_params *p, const void *in, uint8_t *packed, size_t 
   memset(packed, 0, (size_t)L.total_bytes);
   write_header(p, &L, packed);
 
-  /* Sec. 3.2: entropy score of every tile, then top-p% per sample. */
+  /* Sec. 3.2: entropy score of every allocation tile (A consecutive channels of one token = m
+   * consecutive quantisation tiles), top-p% of them per sample, and the chosen width for every
+   * quantisation tile inside. */
   uint8_t *is_hi = (uint8_t *)calloc((size_t)n, 1);
   if (L.k_hi > 0) {
-    float *score = (float *)malloc((size_t)n * sizeof(float));
+    const uint32_t A = p->alloc_tile ? p->alloc_tile : G;
+    const uint64_t m = A / G, na = n / m, nag = ng / m;
+    float *score = (float *)malloc((size_t)na * sizeof(float));
+    uint8_t *a_hi = (uint8_t *)calloc((size_t)na, 1);
 #pragma omp parallel for schedule(static)
-    for (int64_t t = 0; t < (int64_t)n; t++) {
-      float x[128];
-      load_tile(p, in, (uint64_t)t, x);
-      score[t] = tahqo_score(x, G, p->eps_l1, p->eps_log);
+    for (int64_t t = 0; t < (int64_t)na; t++) {
+      float *x = (float *)malloc((size_t)A * sizeof(float));
+      for (uint64_t j = 0; j < m; j++) load_tile(p, in, (uint64_t)t * m + j, x + j * G);
+      score[t] = tahqo_score(x, A, p->eps_l1, p->eps_log);
+      free(x);
     }
 #pragma omp parallel for schedule(static)
     for (int64_t g = 0; g < (int64_t)L.n_groups; g++)
-      tahqo_allocate(score + (uint64_t)g * ng, ng, L.k_hi, is_hi + (uint64_t)g * ng);
+      tahqo_allocate(score + (uint64_t)g * nag, nag, L.k_hi / m, a_hi + (uint64_t)g * nag);
+    for (uint64_t t = 0; t < n; t++) is_hi[t] = a_hi[t / m];
+    free(a_hi);
     free(score);
   }
 

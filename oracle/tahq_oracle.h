@@ -38,11 +38,13 @@ typedef struct {
   float eps_ratio;           /* varrho of Eq. 3                                                    */
   uint32_t rounding;         /* 0 = round-half-even, 1 = stochastic (Philox4x32-10)                */
   uint64_t seed;             /* key of the stochastic-rounding stream                              */
+  uint32_t alloc_tile;       /* A of Sec. 3.2: allocation-tile width, a multiple of tile that divides
+                                hidden; 0 means A = G (the paper's default); A = hidden is token-level   */
 } tahqo_params;
 
 /* Section offsets of the packed buffer (bytes from its start). */
 typedef struct {
-  uint64_t n_tiles, n_groups, tiles_per_group, k_hi;
+  uint64_t n_tiles, n_groups, tiles_per_group, k_hi;   /* k_hi counts quantisation tiles per group */
   uint32_t lo_bits, hi_bits;
   uint64_t off_bitmap, off_scale_zero, off_pivot, off_payload;
   uint64_t payload_bytes, total_bytes;
@@ -57,7 +59,7 @@ int tahqo_encode(const tahqo_params *p, const void *in, uint8_t *packed, size_t 
 int tahqo_decode(const tahqo_params *p, const uint8_t *packed, size_t packed_bytes, void *out);
 
 /* Per-step entry points, exported so that the tests can pin each step alone. */
-float tahqo_treesum(const float *x, uint32_t n);                       /* fixed pairwise tree      */
+float tahqo_treesum(const float *x, uint32_t n);                       /* fixed pairwise tree, any n */
 void tahqo_lg2_array(const float *x, float *y, size_t n);             /* the oracle's log2        */
 float tahqo_score(const float *tile, uint32_t G, float eps_l1, float eps_log); /* Eq. 1-2         */
 void tahqo_allocate(const float *score, uint64_t n, uint64_t k_hi, uint8_t *is_hi); /* Sec. 3.2   */

@@ -299,3 +299,69 @@ def test_stochastic_mode_whole_tensor_is_unbiased():
     p0 = O.Params(tokens=16, hidden=256, group_tokens=16, budget_millibits=3000, tau=float("inf"))
     det = O.decode(p0, O.encode(p0, x))
     assert relerr(acc / n, x) < 0.1 * relerr(det, x)
+
+
+# ---------------------------------------------------------------- allocation tiles wider than quantisation tiles (Sec. 3.2)
+def _shannon64(v):
+    a = np.abs(v.astype(np.float64))
+    p = a / (a.sum() + 1e-8)
+    return float(-(p * np.log2(p + 1e-8)).sum())
+
+
+def _bitmap(p, buf):
+    L = O.layout(p)
+    return np.unpackbits(buf[L["off_bitmap"]:L["off_bitmap"] + (L["n_tiles"] + 7) // 8], bitorder="little")[:L["n_tiles"]]
+
+
+def test_tree_sum_of_any_length():
+    """A partial sum without a neighbour waits for the next level: n = 3 -> (x0+x1)+x2, n = 6 -> ((x0+x1)+(x2+x3))+(x4+x5)."""
+    f = np.float32
+    x = np.array([1e8, 1.0, -1e8, 3.0, 5.0, 7.0], dtype=np.float32)
+    assert O.treesum(x[:3]) == f(f(x[0] + x[1]) + x[2])
+    assert O.treesum(x) == f(f(f(x[0] + x[1]) + f(x[2] + x[3])) + f(x[4] + x[5]))
+    y = np.arange(1, 13, dtype=np.float32)
+    assert O.treesum(y) == 78.0
+    # 768 = 3 * 256: three power-of-two blocks, ((b0 + b1) + b2)
+    z = np.random.default_rng(1).standard_normal(768).astype(np.float32)
+    b = [O.treesum(z[i * 256:(i + 1) * 256]) for i in range(3)]
+    assert O.treesum(z) == f(f(b[0] + b[1]) + b[2])
+
+
+@pytest.mark.parametrize("hidden,G,A", [(256, 64, 128), (256, 64, 256), (768, 64, 192), (768, 64, 768), (512, 32, 128)])
+def test_allocation_tile_wider_than_quantisation_tile(hidden, G, A):
+    """A = m*G: the entropy is taken over A channels, the top-p% of the S*C/A allocation tiles of a sample get
+    the higher width, and all m quantisation tiles inside share it; A = C is token-level allocation."""
+    rng = np.random.default_rng(hidden + A)
+    S, B = 16, 3
+    x = (rng.standard_normal((B * S, hidden)) * np.exp(rng.standard_normal((B * S, 1)))).astype(np.float32)
+    x[:, ::53] *= 20
+    p = O.Params(tokens=B * S, hidden=hidden, group_tokens=S, tile=G, budget_millibits=3500, alloc_tile=A)
+    L = O.layout(p)
+    m, na_g = A // G, S * (hidden // A)
+    k_a = na_g * 500 // 1000
+    assert L["k_hi"] == k_a * m
+    assert L["payload_bytes"] == B * (G // 8) * (L["tiles_per_group"] * 3 + L["k_hi"])
+    buf = O.encode(p, x)
+    bm = _bitmap(p, buf).reshape(B, na_g, m)
+    assert (bm.min(axis=2) == bm.max(axis=2)).all()                 # one width per allocation tile
+    assert (bm[:, :, 0].sum(axis=1) == k_a).all()                   # exactly the top-p% per sample
+    # which ones: the float64 Shannon entropy over A channels, wherever the ranking is not a near-tie
+    tiles = x.reshape(B, na_g, A)
+    for b in range(B):
+        h = np.array([_shannon64(t) for t in tiles[b]])
+        order = np.argsort(-h, kind="stable")
+        if k_a and k_a < na_g and h[order[k_a - 1]] - h[order[k_a]] > 1e-4:
+            assert set(np.flatnonzero(bm[b, :, 0])) == set(order[:k_a])
+    # decode still inverts it, and the header tells the two apart
+    y = O.decode(p, buf)
+    assert np.abs(y - x).max() <= np.abs(x).max()
+    assert int(buf[88:92].view(np.uint32)[0]) == A
+
+
+def test_default_allocation_tile_is_the_quantisation_tile():
+    x = np.random.default_rng(5).standard_normal((32, 256)).astype(np.float32)
+    a = O.encode(O.Params(tokens=32, hidden=256, group_tokens=16, tile=64, budget_millibits=3800), x)
+    b = O.encode(O.Params(tokens=32, hidden=256, group_tokens=16, tile=64, budget_millibits=3800, alloc_tile=64), x)
+    assert np.array_equal(a, b)
+    for bad in (96, 48, 512):
+        assert O.packed_bound(O.Params(tokens=32, hidden=256, group_tokens=16, tile=64, alloc_tile=bad)) == 0
