@@ -83,6 +83,12 @@ typedef struct {
                                 of Philox4x32-10(key = seed, counter = i / 4) times 2^-24, i = the
                                 element's index in the tensor: codes are a function of (input, seed)  */
   uint64_t seed;             /* used only when rounding == 1                                     */
+  uint32_t alloc_tile;       /* A of Sec. 3.2: allocation-tile width, a multiple of tile that divides
+                                hidden and is at most 8192; 0 = tile (the paper's default).  The entropy
+                                is taken over A channels, the top-p% of the S*hidden/A allocation tiles of
+                                a ranking group get the higher width, and every quantisation tile inside
+                                shares it; A = hidden is token-level allocation.  A != tile needs tile 32
+                                or 64 (TAHQ_ERR_UNSUPPORTED otherwise).                              */
 } tahq_params;
 
 /* Byte offsets of the sections of the packed buffer (all multiples of 128). */

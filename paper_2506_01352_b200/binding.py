@@ -24,7 +24,7 @@ class _Params(C.Structure):
         ("struct_size", C.c_uint32), ("dtype", C.c_uint32), ("tokens", C.c_uint64), ("hidden", C.c_uint32),
         ("group_tokens", C.c_uint32), ("tile", C.c_uint32), ("budget_millibits", C.c_uint32),
         ("tau", C.c_float), ("eps_l1", C.c_float), ("eps_log", C.c_float), ("eps_ratio", C.c_float),
-        ("rounding", C.c_uint32), ("seed", C.c_uint64),
+        ("rounding", C.c_uint32), ("seed", C.c_uint64), ("alloc_tile", C.c_uint32),
     ]
 
 
@@ -53,11 +53,12 @@ class Params:
     eps_ratio: float = 1e-8
     rounding: int = 0
     seed: int = 0
+    alloc_tile: int = 0
 
     def c(self) -> _Params:
         return _Params(C.sizeof(_Params), self.dtype, self.tokens, self.hidden, self.group_tokens, self.tile,
                        self.budget_millibits, self.tau, self.eps_l1, self.eps_log, self.eps_ratio,
-                       self.rounding, self.seed)
+                       self.rounding, self.seed, self.alloc_tile)
 
 
 class TahqError(RuntimeError):

@@ -44,6 +44,8 @@ struct Plan {
   bool mixed;             // two widths in use (k_hi > 0)
   bool direct;            // small ranking groups: select straight from the scores
   uint32_t cpg, cand_cap;
+  uint32_t alloc_m;            // quantisation tiles per allocation tile (Sec. 3.2; 1 by default)
+  uint64_t rank_per_group, rank_k;   // allocation tiles per ranking group, and how many of them get the higher width
   // workspace offsets
   uint64_t ws_flags, ws_ncand, ws_done, ws_nabove, ws_hist, ws_zero_end, ws_scores, ws_theta, ws_cand, ws_total;
 };
@@ -78,6 +80,9 @@ static tahq_status make_plan(const tahq_params *p, Plan *pl) {
     return TAHQ_ERR_INVALID_ARG;
   const uint64_t M = p->hidden / G;
   if (p->tokens > (1ull << 40) / M) return TAHQ_ERR_INVALID_ARG;
+  const uint32_t A = p->alloc_tile ? p->alloc_tile : G;   // allocation-tile width (Sec. 3.2)
+  if (A % G || A > p->hidden || p->hidden % A) return TAHQ_ERR_INVALID_ARG;
+  pl->alloc_m = A / G;
   tahq_layout &L = pl->L;
   L.n_tiles = p->tokens * M;
   L.tiles_per_group = S * M;
@@ -87,7 +92,9 @@ static tahq_status make_plan(const tahq_params *p, Plan *pl) {
   pl->f = beta % 1000;
   L.lo_bits = beta / 1000;
   L.hi_bits = pl->f ? L.lo_bits + 1 : L.lo_bits;
-  L.k_hi = L.tiles_per_group * (uint64_t)pl->f / 1000u;
+  pl->rank_per_group = L.tiles_per_group / pl->alloc_m;
+  pl->rank_k = pl->rank_per_group * (uint64_t)pl->f / 1000u;
+  L.k_hi = pl->rank_k * pl->alloc_m;
   L.payload_bytes = L.n_groups * (uint64_t)(G / 8) * (L.tiles_per_group * L.lo_bits + L.k_hi);
   L.off_bitmap = 128;
   L.off_scale_zero = up(L.off_bitmap + (L.n_tiles + 7) / 8, 128);
@@ -95,17 +102,18 @@ static tahq_status make_plan(const tahq_params *p, Plan *pl) {
   L.off_payload = up(L.off_pivot + L.n_tiles, 128);
   L.total_bytes = up(L.off_payload + L.payload_bytes, 128);
   if (G < 32) return TAHQ_ERR_UNSUPPORTED;
+  if (pl->alloc_m > 1 && (G == 128 || A > 8192)) return TAHQ_ERR_UNSUPPORTED;
 
   pl->mixed = L.k_hi > 0;
-  pl->direct = L.tiles_per_group <= (uint64_t)kSortCap;
+  pl->direct = pl->rank_per_group <= (uint64_t)kSortCap;
   pl->cpg = 1;
   pl->cand_cap = 0;
   if (pl->mixed && !pl->direct) {
-    pl->cpg = (uint32_t)((L.tiles_per_group + kSelSlice - 1) / kSelSlice);
+    pl->cpg = (uint32_t)((pl->rank_per_group + kSelSlice - 1) / kSelSlice);
     // select_kernel copes with more candidates than the list holds; the single-launch encode does not, so
     // there the list holds a whole group (every tile is a candidate when all scores are equal)
     const uint64_t cap = fused_encode_wanted() ? 0xffffffffull : 32768ull;
-    pl->cand_cap = (uint32_t)(L.tiles_per_group < cap ? L.tiles_per_group : cap);
+    pl->cand_cap = (uint32_t)(pl->rank_per_group < cap ? pl->rank_per_group : cap);
   }
   const bool hist = pl->mixed && !pl->direct;
   uint64_t o = 256;                                         // status word and friends
@@ -115,7 +123,7 @@ static tahq_status make_plan(const tahq_params *p, Plan *pl) {
   pl->ws_nabove = o; o = up(o + (hist ? 4 * L.n_groups : 0), 256);
   pl->ws_hist = o;   o += hist ? 4ull * kBins * L.n_groups : 0;
   pl->ws_zero_end = o;                                      // [0, ws_zero_end) is cleared by every encode
-  pl->ws_scores = o; o = up(o + (pl->mixed ? 4 * L.n_tiles : 0), 256);
+  pl->ws_scores = o; o = up(o + (pl->mixed ? 4 * (L.n_tiles / pl->alloc_m) : 0), 256);
   pl->ws_theta = o;  o = up(o + (pl->mixed ? 8 * L.n_groups : 0), 256);
   pl->ws_cand = o;   o = up(o + 8ull * pl->cand_cap * L.n_groups, 256);
   pl->ws_total = o;
@@ -124,6 +132,7 @@ static tahq_status make_plan(const tahq_params *p, Plan *pl) {
 
 static void fill_header(const tahq_params *p, const Plan &pl, uint32_t *h) {
   std::memset(h, 0, 128);
+  h[22] = pl.alloc_m > 1 ? pl.alloc_m * p->tile : 0u;   // allocation-tile width when it is not the tile
   auto f2u = [](float f) { uint32_t u; std::memcpy(&u, &f, 4); return u; };
   auto put64 = [&](int w, uint64_t v) { h[w] = (uint32_t)v; h[w + 1] = (uint32_t)(v >> 32); };
   h[0] = 0x51484154u;  // "TAHQ"
@@ -150,6 +159,9 @@ static void fill_args(const tahq_params *p, const Plan &pl, uint8_t *ws, Args *a
   a->n_tiles = pl.L.n_tiles;
   a->tiles_per_group = pl.L.tiles_per_group;
   a->k_hi = pl.L.k_hi;
+  a->rank_per_group = pl.rank_per_group;
+  a->rank_k = pl.rank_k;
+  a->alloc_m = pl.alloc_m;
   a->n_groups = pl.L.n_groups;
   a->lo = pl.L.lo_bits;
   a->mixed = pl.mixed;
@@ -180,7 +192,7 @@ static void fill_args(const tahq_params *p, const Plan &pl, uint8_t *ws, Args *a
   a->cpg = pl.cpg;
   a->direct = pl.direct;
   // the screening score leaves varsigma out; its share of the score is below G * varsigma / ln 2
-  a->exact_scores = pl.direct || (double)p->tile * (double)p->eps_log > 1e-5;
+  a->exact_scores = pl.direct || pl.alloc_m > 1 || (double)p->tile * (double)p->eps_log > 1e-5;
   fill_header(p, pl, a->header);
 }
 
@@ -260,7 +272,7 @@ static tahq_status encode_t(const Plan &pl, const Args &a_in, cudaStream_t st) {
     // large ranking groups, on request: the whole encode as one cooperative launch (grid-wide barriers
     // between scoring, the exact re-scoring near each group's threshold, and quantise + pack); if the device
     // cannot keep the grid resident the three-kernel path below does the same work
-    if (pl.mixed && !pl.direct && fused_encode_wanted()) {
+    if (pl.mixed && !pl.direct && pl.alloc_m == 1 && fused_encode_wanted()) {
       const int smem = StreamCfg<C>::smem_bytes(2);
       const int occ = prepare(encode_fused_kernel<C, SR>, smem, d, occ_fused);
       if (occ) {
@@ -279,8 +291,17 @@ static tahq_status encode_t(const Plan &pl, const Args &a_in, cudaStream_t st) {
       }
     }
   }
+  if (pl.mixed && pl.alloc_m > 1) {   // Sec. 3.2 with A = m * G: one warp per allocation tile, exact scores
+    const uint64_t n_alloc = a.n_tiles / pl.alloc_m;
+    const uint64_t want = (n_alloc + kWarps - 1) / kWarps, cap = (uint64_t)d.sms * 8;
+    const unsigned grid = (unsigned)(want < cap ? want : cap);
+    if (C::BF16) TAHQ_LAUNCH("alloc_score", st, alloc_score_kernel<true><<<grid, kThreads, 0, st>>>(a));
+    else TAHQ_LAUNCH("alloc_score", st, alloc_score_kernel<false><<<grid, kThreads, 0, st>>>(a));
+  }
   if (pl.mixed) {
-    if constexpr (C::LPT == 1) {
+    if (pl.alloc_m > 1) {
+      // scores are in place
+    } else if constexpr (C::LPT == 1) {
       constexpr int NS = C::ROWB <= 128 ? 3 : 2;
       const int smem = kWarps * NS * StreamCfg<C>::UNIT_BYTES + 256;   // ring slots, then the warps' mbarriers
       const int occ = prepare(stats_stream_kernel<C, NS>, smem, d, occ_stats);

@@ -21,6 +21,10 @@ struct Args {
   uint8_t *packed;          // packed buffer (decode reads it)
   uint8_t *out;             // decode: tensor
   uint64_t n_tiles, tiles_per_group, k_hi, n_groups;
+  // Sec. 3.2 ranks allocation tiles: alloc_m quantisation tiles each (1 by default); a ranking group has
+  // rank_per_group of them, the rank_k highest-scoring get the higher width; scores[] has one entry each
+  uint64_t rank_per_group, rank_k;
+  uint32_t alloc_m;
   uint32_t lo, mixed;       // low width; 1 when two widths are in use
   uint64_t off_bitmap, off_sz, off_pivot, off_payload, payload_bytes, total_bytes;
   float tau, eps_l1, eps_log, eps_ratio;
@@ -193,6 +197,76 @@ __global__ void __launch_bounds__(kThreads, 2) stats_kernel(const Args a) {
 }
 
 // ------------------------------------------------------------------------------------------
+// Eq. 1-2 over allocation tiles wider than the quantisation tile (Sec. 3.2, A = m * G, up to 8192
+// channels): one warp per allocation tile, exact arithmetic in the summation order of the pairwise tree
+// -- eight consecutive elements inside a lane, then neighbouring lanes (a lane without a neighbour
+// waits for the next level), then the sums of successive rounds of 256 elements in the same way.
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ float warp_tree(float x, uint32_t n, int lane) {   // n <= 32 values, one per lane
+#pragma unroll
+  for (int h = 1; h < 32; h *= 2) {
+    const float y = __shfl_down_sync(kFull, x, h);
+    if ((lane & (2 * h - 1)) == 0 && (uint32_t)(lane + h) < n) x = x + y;
+  }
+  return __shfl_sync(kFull, x, 0);
+}
+template <bool BF16, class F>
+__device__ __forceinline__ float alloc_tree(const uint8_t *base, uint32_t n_oct, int lane, F &&f) {
+  const uint32_t rounds = (n_oct + 31) / 32;
+  float rs = 0.0f;   // lane r keeps the sum of round r
+  for (uint32_t r = 0; r < rounds; ++r) {
+    const uint32_t o = r * 32 + lane, left = n_oct - r * 32;
+    float v[8];
+    if (o < n_oct) {
+      if constexpr (BF16) {
+        const uint4 w = __ldg(reinterpret_cast<const uint4 *>(base) + o);
+        const uint32_t u[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          v[2 * j] = fabsf(__uint_as_float(u[j] << 16));
+          v[2 * j + 1] = fabsf(__uint_as_float(u[j] & 0xffff0000u));
+        }
+      } else {
+        const float4 p = __ldg(reinterpret_cast<const float4 *>(base) + 2 * o);
+        const float4 q = __ldg(reinterpret_cast<const float4 *>(base) + 2 * o + 1);
+        v[0] = fabsf(p.x); v[1] = fabsf(p.y); v[2] = fabsf(p.z); v[3] = fabsf(p.w);
+        v[4] = fabsf(q.x); v[5] = fabsf(q.y); v[6] = fabsf(q.z); v[7] = fabsf(q.w);
+      }
+#pragma unroll
+      for (int k = 0; k < 8; ++k) v[k] = f(v[k]);
+    } else {
+#pragma unroll
+      for (int k = 0; k < 8; ++k) v[k] = 0.0f;
+    }
+    const float x = warp_tree(tree8(v), left < 32 ? left : 32u, lane);
+    if ((uint32_t)lane == r) rs = x;
+  }
+  return warp_tree(rs, rounds, lane);
+}
+template <bool BF16>
+__global__ void __launch_bounds__(kThreads) alloc_score_kernel(const Args a) {
+  const int lane = threadIdx.x & 31;
+  const uint64_t warp = ((uint64_t)blockIdx.x * kThreads + threadIdx.x) >> 5;
+  const uint64_t n_warps = ((uint64_t)gridDim.x * kThreads) >> 5;
+  const uint32_t A = a.alloc_m * a.tile, n_oct = A / 8;
+  const uint64_t n_alloc = a.n_tiles / a.alloc_m;
+  for (uint64_t t = warp; t < n_alloc; t += n_warps) {
+    const uint8_t *base = a.in + t * (uint64_t)A * (BF16 ? 2 : 4);
+    const float L1 = alloc_tree<BF16>(base, n_oct, lane, [](float m) { return m; });
+    const float inv = __fdiv_rn(1.0f, L1 + a.eps_l1);
+    const float S = alloc_tree<BF16>(base, n_oct, lane, [&](float m) {
+      const float p = m * inv;
+      return p * lg2_fma(p + a.eps_log);
+    });
+    if (lane == 0) {
+      const float sc = 0.0f - S;
+      a.scores[t] = sc;
+      if (!a.direct) atomicAdd(a.hist + (t / a.rank_per_group) * kBins + score_bin(sc), 1u);
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------
 // Sec. 3.2: exact top-k_hi per ranking group -> theta[g], the ranking key of the k_hi-th tile
 // ------------------------------------------------------------------------------------------
 constexpr int kSelThreads = 1024;
@@ -276,7 +350,7 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const Args a) {
   __shared__ uint32_t s_sel[2];
   __shared__ uint32_t s_last;
   const uint64_t g = blockIdx.x / a.cpg;
-  const uint64_t ng = a.tiles_per_group;
+  const uint64_t ng = a.rank_per_group;
   const float *sc = a.scores + g * ng;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   auto from_smem = [&](uint64_t i, unsigned long long &key) { key = s_keys[i]; return true; };
@@ -284,7 +358,7 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const Args a) {
   if (a.direct) {   // small group: rank all of its tiles here (one CTA per group)
     for (uint32_t i = threadIdx.x; i < (uint32_t)ng; i += kSelThreads) s_keys[i] = rank_key(sc[i], i);
     __syncthreads();
-    const unsigned long long t = radix_select(ng, (uint32_t)a.k_hi, from_smem);
+    const unsigned long long t = radix_select(ng, (uint32_t)a.rank_k, from_smem);
     if (threadIdx.x == 0) a.theta[g] = t;
     return;
   }
@@ -314,7 +388,7 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const Args a) {
   __syncthreads();
   uint32_t above = incl - mine;
   for (int w = warp + 1; w < kSelThreads / 32; ++w) above += s_warp[w];
-  const uint32_t k = (uint32_t)a.k_hi;
+  const uint32_t k = (uint32_t)a.rank_k;
   if (above < k && above + mine >= k) {
 #pragma unroll
     for (int j = BPT - 1; j >= 0; --j) {
@@ -374,7 +448,9 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const Args a) {
       const uint64_t i = lo + s_list[live ? j : 0];
       const uint8_t *tp = a.in + (g * ng + i) * (uint64_t)tile_bytes;
       float ex;
-      if (a.bf16) {
+      if (a.exact_scores) {   // nothing to recompute (and with wider allocation tiles tp is not the tile)
+        ex = scw[i];
+      } else if (a.bf16) {
         ex = noct == 4   ? exact_score_coop<4, true>(tp, sub, a.eps_l1, a.eps_log)
              : noct == 8 ? exact_score_coop<8, true>(tp, sub, a.eps_l1, a.eps_log)
                          : exact_score_coop<16, true>(tp, sub, a.eps_l1, a.eps_log);
@@ -399,8 +475,8 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const Args a) {
   __threadfence();
   const uint32_t n = *reinterpret_cast<volatile uint32_t *>(a.ncand + g);
   const uint32_t nab = *reinterpret_cast<volatile uint32_t *>(a.nabove + g);
-  uint32_t rr = (uint32_t)a.k_hi - nab;   // rank of the threshold tile among the candidates
-  if (nab >= (uint32_t)a.k_hi || rr > n) {   // only possible if the screening error exceeded its bound
+  uint32_t rr = (uint32_t)a.rank_k - nab;   // rank of the threshold tile among the candidates
+  if (nab >= (uint32_t)a.rank_k || rr > n) {   // only possible if the screening error exceeded its bound
     if (threadIdx.x == 0) atomicOr(a.status, 8u /* TAHQ_DEV_INTERNAL */);
     rr = rr > n ? n : 1u;
     if (n == 0) { if (threadIdx.x == 0) a.theta[g] = ~0ull; return; }
@@ -460,6 +536,7 @@ struct GroupCursor {
     uint64_t gg = g;
     uint64_t i = (uint64_t)rem + off;
     if (i >= a.tiles_per_group) { gg += i / a.tiles_per_group; i %= a.tiles_per_group; }
+    if (a.alloc_m > 1) { tile /= a.alloc_m; i /= a.alloc_m; }   // the allocation tile this one lies in
     if constexpr (COH) return rank_key(__ldcg(a.scores + tile), (uint32_t)i) >= __ldcg(a.theta + gg);
     else return rank_key(__ldg(a.scores + tile), (uint32_t)i) >= __ldg(a.theta + gg);
   }

@@ -641,7 +641,7 @@ __device__ __forceinline__ void screen_group(const Args &a, uint64_t g, uint64_t
   __syncthreads();
   uint32_t above = incl - mine;
   for (int w = warp + 1; w < kWarps; ++w) above += s_warp[w];
-  const uint32_t k = (uint32_t)a.k_hi;
+  const uint32_t k = (uint32_t)a.rank_k;
   if (above < k && above + mine >= k) {
 #pragma unroll
     for (int j = BPT - 1; j >= 0; --j) {
@@ -705,8 +705,8 @@ __device__ __forceinline__ void screen_group(const Args &a, uint64_t g, uint64_t
 // tiles of the group computes it for itself and stores it (all of them the same value).
 __device__ __forceinline__ void rank_group(const Args &a, uint64_t g, unsigned long long *s_keys /* 1024 */) {
   const uint32_t n = __ldcg(a.ncand + g), nab = __ldcg(a.nabove + g);
-  uint32_t rr = (uint32_t)a.k_hi - nab;   // rank of the threshold tile among the candidates
-  if (nab >= (uint32_t)a.k_hi || rr > n || n > a.cand_cap) {   // only possible if the screening bound was violated
+  uint32_t rr = (uint32_t)a.rank_k - nab;   // rank of the threshold tile among the candidates
+  if (nab >= (uint32_t)a.rank_k || rr > n || n > a.cand_cap) {   // only possible if the screening bound was violated
     if (threadIdx.x == 0) atomicOr(a.status, 8u /* TAHQ_DEV_INTERNAL */);
     rr = rr > n ? n : 1u;
     if (n == 0 || n > a.cand_cap) {

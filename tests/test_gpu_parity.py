@@ -16,7 +16,7 @@ pytestmark = pytest.mark.gpu
 def oparams(p: T.Params) -> O.Params:
     return O.Params(tokens=p.tokens, hidden=p.hidden, dtype=p.dtype, group_tokens=p.group_tokens, tile=p.tile,
                     budget_millibits=p.budget_millibits, tau=p.tau, eps_l1=p.eps_l1, eps_log=p.eps_log,
-                    eps_ratio=p.eps_ratio, rounding=p.rounding, seed=p.seed)
+                    eps_ratio=p.eps_ratio, rounding=p.rounding, seed=p.seed, alloc_tile=p.alloc_tile)
 
 
 def sections(p: T.Params, buf: np.ndarray):
@@ -234,6 +234,28 @@ def test_fused_cooperative_encode_matches_too():
     root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
     r = subprocess.run([sys.executable, "-c", code], cwd=root, env=env, capture_output=True, text=True, timeout=600)
     assert r.returncode == 0 and "fused ok" in r.stdout, r.stdout + r.stderr
+
+
+@pytest.mark.parametrize("name,S,G,A", [("c1_tiny", 64, 64, 128), ("c1_tiny", 64, 64, 256), ("c1_tiny", 64, 32, 128),
+                                        ("c2_gpt2s", 1024, 64, 192), ("c2_gpt2s", 1024, 64, 768),
+                                        ("c3_llama7b", 2048, 64, 256), ("c3_llama7b", 2048, 64, 4096),
+                                        ("c3_llama7b", 2048, 32, 2048)])
+def test_allocation_tile_wider_than_quantisation_tile(name, S, G, A):
+    """A = m*G (Sec. 3.2): entropy over A channels, top-p% of the allocation tiles per sample, one width per
+    allocation tile; A = hidden is token-level allocation.  Small and large ranking groups, m a power of two or not."""
+    x = synth.make(name, device="cuda")
+    for beta in (3800, 2500):
+        p = T.params_for(x, group_tokens=S, tile=G, budget_millibits=beta, alloc_tile=A)
+        packed, want, ws = check_encode(p, x)
+        check_decode(p, packed, want, ws)
+
+
+def test_allocation_tile_limits():
+    x = synth.make("c1_tiny", device="cuda")
+    assert T.packed_bound(T.params_for(x, group_tokens=64, tile=64, alloc_tile=96)) == 0          # not a multiple of the tile
+    assert T.packed_bound(T.params_for(x, group_tokens=64, tile=128, alloc_tile=256)) == 0        # 128-wide tiles: not built
+    assert T.packed_bound(T.params_for(x, group_tokens=64, tile=64, alloc_tile=64)) == \
+        T.packed_bound(T.params_for(x, group_tokens=64, tile=64))
 
 
 def test_decode_refuses_a_foreign_buffer():
