@@ -37,7 +37,7 @@ typedef struct CUstream_st *tahq_stream;
 typedef enum {
   TAHQ_OK = 0,
   TAHQ_ERR_INVALID_ARG = 1,      /* null pointer, bad struct_size, bad shape/tile/budget        */
-  TAHQ_ERR_UNSUPPORTED = 2,      /* valid in the format but not built (tile < 32)               */
+  TAHQ_ERR_UNSUPPORTED = 2,      /* valid in the format but not built (see alloc_tile)          */
   TAHQ_ERR_BUFFER_TOO_SMALL = 3, /* packed_cap / packed_bytes / ws_cap below the bound          */
   TAHQ_ERR_MISALIGNED = 4,       /* a device pointer is not 16-byte aligned                     */
   TAHQ_ERR_CUDA = 5,             /* a CUDA runtime call (launch, memset) failed                 */
@@ -67,7 +67,8 @@ typedef struct {
   uint64_t tokens;           /* T = B*S                                                          */
   uint32_t hidden;           /* C, a multiple of tile                                            */
   uint32_t group_tokens;     /* S; 0 = the whole tensor is one ranking group; must divide T      */
-  uint32_t tile;             /* G in {32, 64, 128}                                               */
+  uint32_t tile;             /* G in {8, 16, 32, 64, 128} (8 and 16: the small groups of the paper's
+                                ablation; their metadata costs 5.1 / 2.6 bits per element)          */
   uint32_t budget_millibits; /* payload bits per element x 1000, in [2000, 8000].  lo = b/1000
                                 bits for every tile, and the floor(n_g*(b%1000)/1000) highest-
                                 entropy tiles of each ranking group get lo+1.  3800 is the

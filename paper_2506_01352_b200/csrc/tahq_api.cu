@@ -101,7 +101,6 @@ static tahq_status make_plan(const tahq_params *p, Plan *pl) {
   L.off_pivot = up(L.off_scale_zero + 4 * L.n_tiles, 128);
   L.off_payload = up(L.off_pivot + L.n_tiles, 128);
   L.total_bytes = up(L.off_payload + L.payload_bytes, 128);
-  if (G < 32) return TAHQ_ERR_UNSUPPORTED;
   if (pl->alloc_m > 1 && (G == 128 || A > 8192)) return TAHQ_ERR_UNSUPPORTED;
 
   pl->mixed = L.k_hi > 0;
@@ -423,12 +422,16 @@ tahq_status tahq_encode(const tahq_params *p, const void *d_in, void *d_packed, 
   const bool bf = p->dtype == TAHQ_BF16;
   if (p->rounding == 1) {   // stochastic rounding: kernels of their own, the default path carries none of it
     switch (p->tile) {
+      case 8: return bf ? encode_t<Cfg<8, true>, true>(pl, a, st) : encode_t<Cfg<8, false>, true>(pl, a, st);
+      case 16: return bf ? encode_t<Cfg<16, true>, true>(pl, a, st) : encode_t<Cfg<16, false>, true>(pl, a, st);
       case 32: return bf ? encode_t<Cfg<32, true>, true>(pl, a, st) : encode_t<Cfg<32, false>, true>(pl, a, st);
       case 64: return bf ? encode_t<Cfg<64, true>, true>(pl, a, st) : encode_t<Cfg<64, false>, true>(pl, a, st);
       default: return bf ? encode_t<Cfg<128, true>, true>(pl, a, st) : encode_t<Cfg<128, false>, true>(pl, a, st);
     }
   }
   switch (p->tile) {
+    case 8: return bf ? encode_t<Cfg<8, true>, false>(pl, a, st) : encode_t<Cfg<8, false>, false>(pl, a, st);
+    case 16: return bf ? encode_t<Cfg<16, true>, false>(pl, a, st) : encode_t<Cfg<16, false>, false>(pl, a, st);
     case 32: return bf ? encode_t<Cfg<32, true>, false>(pl, a, st) : encode_t<Cfg<32, false>, false>(pl, a, st);
     case 64: return bf ? encode_t<Cfg<64, true>, false>(pl, a, st) : encode_t<Cfg<64, false>, false>(pl, a, st);
     default: return bf ? encode_t<Cfg<128, true>, false>(pl, a, st) : encode_t<Cfg<128, false>, false>(pl, a, st);
@@ -452,6 +455,8 @@ tahq_status tahq_decode(const tahq_params *p, const void *d_packed, size_t packe
   if (cudaMemsetAsync(d_ws, 0, pl.ws_ncand, st) != cudaSuccess) return TAHQ_ERR_CUDA;   // status + flags
   const bool bf = p->dtype == TAHQ_BF16;
   switch (p->tile) {
+    case 8: return bf ? decode_t<Cfg<8, true>>(pl, a, st) : decode_t<Cfg<8, false>>(pl, a, st);
+    case 16: return bf ? decode_t<Cfg<16, true>>(pl, a, st) : decode_t<Cfg<16, false>>(pl, a, st);
     case 32: return bf ? decode_t<Cfg<32, true>>(pl, a, st) : decode_t<Cfg<32, false>>(pl, a, st);
     case 64: return bf ? decode_t<Cfg<64, true>>(pl, a, st) : decode_t<Cfg<64, false>>(pl, a, st);
     default: return bf ? decode_t<Cfg<128, true>>(pl, a, st) : decode_t<Cfg<128, false>>(pl, a, st);

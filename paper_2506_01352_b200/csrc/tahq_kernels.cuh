@@ -451,11 +451,15 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const Args a) {
       if (a.exact_scores) {   // nothing to recompute (and with wider allocation tiles tp is not the tile)
         ex = scw[i];
       } else if (a.bf16) {
-        ex = noct == 4   ? exact_score_coop<4, true>(tp, sub, a.eps_l1, a.eps_log)
+        ex = noct == 1   ? exact_score_coop<1, true>(tp, sub, a.eps_l1, a.eps_log)
+             : noct == 2 ? exact_score_coop<2, true>(tp, sub, a.eps_l1, a.eps_log)
+             : noct == 4 ? exact_score_coop<4, true>(tp, sub, a.eps_l1, a.eps_log)
              : noct == 8 ? exact_score_coop<8, true>(tp, sub, a.eps_l1, a.eps_log)
                          : exact_score_coop<16, true>(tp, sub, a.eps_l1, a.eps_log);
       } else {
-        ex = noct == 4   ? exact_score_coop<4, false>(tp, sub, a.eps_l1, a.eps_log)
+        ex = noct == 1   ? exact_score_coop<1, false>(tp, sub, a.eps_l1, a.eps_log)
+             : noct == 2 ? exact_score_coop<2, false>(tp, sub, a.eps_l1, a.eps_log)
+             : noct == 4 ? exact_score_coop<4, false>(tp, sub, a.eps_l1, a.eps_log)
              : noct == 8 ? exact_score_coop<8, false>(tp, sub, a.eps_l1, a.eps_log)
                          : exact_score_coop<16, false>(tp, sub, a.eps_l1, a.eps_log);
       }
@@ -594,7 +598,11 @@ constexpr float kMagic = 12582912.0f;   // 1.5 * 2^23: adding it rounds to the n
 
 template <class C>
 __device__ __forceinline__ constexpr float hadamard_scale() {
-  return (C::G == 32) ? 0.17677669529663687f : (C::G == 64) ? 0.125f : 0.08838834764831845f;
+  return (C::G == 8)    ? 0.35355339059327379f
+         : (C::G == 16) ? 0.25f
+         : (C::G == 32) ? 0.17677669529663687f
+         : (C::G == 64) ? 0.125f
+                        : 0.08838834764831845f;
 }
 
 // Range of a row -> binary16 zero-point and scale, and the reciprocal the codes are computed with.
@@ -761,6 +769,58 @@ __device__ __forceinline__ void pack_store_narrow(F &&t, uint32_t W, uint32_t *d
 #pragma unroll
       for (int j = 0; j < NG / 2; ++j) dst[j] = w[j];
     }
+  }
+}
+
+// Tiles of 8 or 16 elements (the small groups of the paper's ablation): a tile's codes are N*W/8 bytes
+// and start on any byte (N = 8) or any even byte (N = 16), so they are assembled as one 128-bit value
+// and leave byte by byte.
+template <int N, class F>
+__device__ __forceinline__ void pack_store_small(F &&t, uint32_t W, uint8_t *dst) {
+  static_assert(N == 8 || N == 16, "small tiles");
+  unsigned long long lo = 0, hi = 0;
+#pragma unroll
+  for (int k = 0; k < N; ++k) {
+    const unsigned long long code = (unsigned long long)(__float_as_uint(t(k)) - 0x4B400000u);
+    const uint32_t pos = (uint32_t)k * W;
+    if (pos < 64) {
+      lo |= code << pos;
+      if (pos + W > 64) hi |= code >> (64 - pos);
+    } else {
+      hi |= code << (pos - 64);
+    }
+  }
+  const uint32_t nbytes = (uint32_t)N * W / 8;
+#pragma unroll
+  for (int j = 0; j < N; ++j)
+    if ((uint32_t)j < nbytes) dst[j] = (uint8_t)(j < 8 ? lo >> (8 * j) : hi >> (8 * (j - 8)));
+}
+
+// ... and back: z + q*s for such a tile (bytes from shared or global memory)
+template <int N>
+__device__ __forceinline__ void dequant_small(const uint8_t *src, uint32_t W, float s, float z, float (&x)[N]) {
+  static_assert(N == 8 || N == 16, "small tiles");
+  unsigned long long lo = 0, hi = 0;
+  const uint32_t nbytes = (uint32_t)N * W / 8;
+#pragma unroll
+  for (int j = 0; j < N; ++j)
+    if ((uint32_t)j < nbytes) {
+      const unsigned long long b = src[j];
+      if (j < 8) lo |= b << (8 * j);
+      else hi |= b << (8 * (j - 8));
+    }
+  const unsigned long long mask = (1ull << W) - 1ull;
+#pragma unroll
+  for (int k = 0; k < N; ++k) {
+    const uint32_t pos = (uint32_t)k * W;
+    unsigned long long c;
+    if (pos < 64) {
+      c = lo >> pos;
+      if (pos + W > 64) c |= hi << (64 - pos);
+    } else {
+      c = hi >> (pos - 64);
+    }
+    x[k] = __fmaf_rn((float)(uint32_t)(c & mask), s, z);
   }
 }
 

@@ -251,7 +251,8 @@ __device__ __forceinline__ uint32_t encode_plain_words(const uint32_t (&w)[C::RO
     }
     stochastic_codes<C::EPT>(d, q.inv_s, q.qmax, seed, first);
     auto tk = [&](int k) { return d[k]; };
-    if (narrow) pack_store_narrow<C::EPT>(tk, bits, dst);
+    if constexpr (C::EPT < 32) pack_store_small<C::EPT>(tk, bits, reinterpret_cast<uint8_t *>(dst));
+    else if (narrow) pack_store_narrow<C::EPT>(tk, bits, dst);
     else pack_row<C::EPT>(tk, bits, dst);
     return q.sz;
   }
@@ -273,7 +274,8 @@ __device__ __forceinline__ uint32_t encode_plain_words(const uint32_t (&w)[C::RO
       t[i] = f2(fminf(fmaxf(t[i].x, kMagic), kMagic + q.qmax), fminf(fmaxf(t[i].y, kMagic), kMagic + q.qmax));
   }
   auto tk = [&](int k) { return (k & 1) ? t[k >> 1].y : t[k >> 1].x; };
-  if (narrow) pack_store_narrow<C::EPT>(tk, bits, dst);   // every width of this call is at most 4 bits
+  if constexpr (C::EPT < 32) pack_store_small<C::EPT>(tk, bits, reinterpret_cast<uint8_t *>(dst));
+  else if (narrow) pack_store_narrow<C::EPT>(tk, bits, dst);   // every width of this call is at most 4 bits
   else pack_row<C::EPT>(tk, bits, dst);
   return q.sz;
 }
@@ -299,7 +301,7 @@ __device__ __noinline__ void encode_queued_row(float tau, float eps_ratio, uint8
   load_row_pairs<C>(queue, row, p);
   // Eq. 4: (1/sqrt G) H_G.  For G = 64 the factor is a power of two: the products are exact, so the
   // factor is applied to the range and inside the quantiser's subtraction instead of element by element.
-  constexpr bool kFold = C::G == 64;
+  constexpr bool kFold = C::G == 64 || C::G == 16;
   if (flag) {
     butterfly2<C::EPT / 2>(p);
     if (!kFold) {
@@ -334,7 +336,8 @@ __device__ __noinline__ void encode_queued_row(float tau, float eps_ratio, uint8
   *sz = q.sz;
   *pv = flag ? (uint8_t)(0x80 | d) : (uint8_t)0;
   auto tk = [&](int k) { return (k & 1) ? p[k >> 1].y : p[k >> 1].x; };
-  if (narrow) pack_store_narrow<C::EPT>(tk, bits, dst);
+  if constexpr (C::EPT < 32) pack_store_small<C::EPT>(tk, bits, reinterpret_cast<uint8_t *>(dst));
+  else if (narrow) pack_store_narrow<C::EPT>(tk, bits, dst);
   else pack_row<C::EPT>(tk, bits, dst);
 }
 
@@ -821,7 +824,9 @@ __device__ __forceinline__ void dequant_narrow(const uint32_t (&wv)[N / 8], uint
 template <class C>
 __device__ __forceinline__ void dequant_row(const uint8_t *src, uint32_t bits, bool narrow, float s, float z,
                                             float (&x)[C::EPT]) {
-  if (narrow) {
+  if constexpr (C::EPT < 32) {
+    dequant_small<C::EPT>(src, bits, s, z, x);
+  } else if (narrow) {
     uint32_t wv[C::EPT / 8];
     if constexpr (C::EPT == 64) {
 #pragma unroll
@@ -852,7 +857,7 @@ __device__ __noinline__ void decode_flagged_row(const uint8_t *codes, uint32_t b
   float z = __half2float(__ushort_as_half((unsigned short)(szw >> 16)));
   // 1/sqrt(G) is a power of two for G = 64: scaling s and z by it beforehand scales every later value
   // by it exactly, so the result has the same bits as multiplying at the end
-  constexpr bool kFold = C::G == 64;
+  constexpr bool kFold = C::G == 64 || C::G == 16;
   if (kFold) { s *= hadamard_scale<C>(); z *= hadamard_scale<C>(); }
   float x[C::EPT];
   dequant_row<C>(codes, bits, narrow, s, z, x);

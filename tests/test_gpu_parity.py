@@ -61,7 +61,7 @@ def check_decode(p: T.Params, packed: torch.Tensor, want_packed: np.ndarray, ws)
                           want.view(np.uint32 if p.dtype == T.F32 else np.uint16))
 
 
-@pytest.mark.parametrize("G", [32, 64, 128])
+@pytest.mark.parametrize("G", [8, 16, 32, 64, 128])
 @pytest.mark.parametrize("beta", [4000, 3800, 3000, 2200, 6000, 8000, 7500])
 def test_c1_tiny(G, beta):
     x = synth.make("c1_tiny", device="cuda")
@@ -70,7 +70,7 @@ def test_c1_tiny(G, beta):
     check_decode(p, packed, want, ws)
 
 
-@pytest.mark.parametrize("G", [32, 64, 128])
+@pytest.mark.parametrize("G", [8, 16, 32, 64, 128])
 def test_c1_tiny_bf16(G):
     x = synth.make("c1_tiny", device="cuda", microbatch=1).to(torch.bfloat16)
     p = T.params_for(x, group_tokens=64, tile=G, budget_millibits=3500)
@@ -104,7 +104,8 @@ def test_c4_llama13b(G, beta):
 
 
 @pytest.mark.parametrize("shape,S,G", [((1, 64), 0, 64), ((1, 32), 1, 32), ((3, 128), 3, 128), ((7, 96), 7, 32),
-                                       ((300, 192), 100, 64), ((513, 640), 171, 128), ((1000, 64), 8, 64)])
+                                       ((300, 192), 100, 64), ((513, 640), 171, 128), ((1000, 64), 8, 64),
+                                       ((5, 8), 5, 8), ((77, 48), 11, 16), ((260, 1000), 0, 8)])
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
 def test_ragged_and_degenerate_shapes(shape, S, G, dtype):
     g = torch.Generator(device="cuda").manual_seed(shape[0] * 1000 + shape[1])
@@ -172,7 +173,7 @@ def test_selection_with_near_tied_scores(eps_log):
     check_decode(p, packed, want, ws)
 
 
-@pytest.mark.parametrize("G", [32, 64, 128])
+@pytest.mark.parametrize("G", [8, 16, 32, 64, 128])
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
 def test_stochastic_rounding_mode(G, dtype):
     """rounding = 1 (not in the paper): floor(y + u) with u from Philox4x32-10 keyed by the seed and indexed by
@@ -256,6 +257,16 @@ def test_allocation_tile_limits():
     assert T.packed_bound(T.params_for(x, group_tokens=64, tile=128, alloc_tile=256)) == 0        # 128-wide tiles: not built
     assert T.packed_bound(T.params_for(x, group_tokens=64, tile=64, alloc_tile=64)) == \
         T.packed_bound(T.params_for(x, group_tokens=64, tile=64))
+
+
+@pytest.mark.parametrize("G,beta", [(8, 3800), (16, 3500), (16, 6000)])
+def test_small_tiles_on_a_large_tensor(G, beta):
+    """The small groups of the paper's ablation (TS = 8, 16) on the LLaMA-7B-shaped tensor: ranking groups of
+    up to a million tiles, codes that start on odd bytes."""
+    x = synth.make("c3_llama7b", device="cuda")[:2048].contiguous()
+    p = T.params_for(x, group_tokens=2048, tile=G, budget_millibits=beta)
+    packed, want, ws = check_encode(p, x)
+    check_decode(p, packed, want, ws)
 
 
 def test_decode_refuses_a_foreign_buffer():
