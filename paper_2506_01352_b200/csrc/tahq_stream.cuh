@@ -949,31 +949,40 @@ __global__ void __launch_bounds__(kThreads, 2) decode_stream_kernel(const Args a
   // cp.async of unit u's codes, scale/zero words and pivot bytes into a slot; `hib` = higher-width tiles
   // of the CTA before the unit.  A unit whose codes would reach past the payload (corrupt bit map) is
   // not fetched.
-  auto unit_range = [&](uint64_t u, uint32_t hib, uint32_t word, uint64_t &off, uint32_t &len) {
-    const uint64_t t0 = u * 32;
-    const uint64_t left = a.n_tiles - t0;
-    const uint32_t nv = left < 32 ? (uint32_t)left : 32u;
-    off = (uint64_t)(C::G / 8) * ((uint64_t)a.lo * t0 + base_hi + hib);
+  // Inside the loops everything is relative to the CTA's first tile and first payload byte (32-bit).
+  // pay_off0 = byte offset of the CTA's first code in the payload, known after the look-back.
+  uint64_t pay_off0 = 0;
+  const uint32_t n_rel = a.n_tiles - tile_cta < 0xffffffffull ? (uint32_t)(a.n_tiles - tile_cta) : 0xffffffffu;
+  // bytes [off, off + len) of the CTA's codes belong to the unit whose first tile is trel0 (relative)
+  auto unit_range = [&](uint32_t trel0, uint32_t hib, uint32_t word, uint32_t &off, uint32_t &len) {
+    const uint32_t left = n_rel - trel0;
+    const uint32_t nv = left < 32u ? left : 32u;
+    off = (uint32_t)(C::G / 8) * (a.lo * trel0 + hib);
     len = (uint32_t)(C::G / 8) * (a.lo * nv + (uint32_t)__popc(word));
-    return off + len <= a.payload_bytes;
+    return pay_off0 + off + len <= a.payload_bytes;   // a corrupt bit map must not lead outside the buffer
   };
-  auto issue = [&](uint64_t u, uint32_t su, uint8_t *slot) {   // su = u - first unit of the segment
-    uint64_t off;
-    uint32_t len;
-    if (unit_range(u, s_pre[su], s_bm[su], off, len)) {
-      const uint8_t *src = payload + (off & ~15ull);
-      const uint32_t npieces = ((uint32_t)(off & 15ull) + len + 15u) >> 4;
-      for (uint32_t i = lane; i < npieces; i += 32) cp_async16(slot + (size_t)i * 16, src + (size_t)i * 16, 16);
-      if (lane < 8) cp_async16(slot + S::PAY + lane * 16, a.packed + a.off_sz + u * 128 + lane * 16, 16);
+  // cp.async of a unit's codes (from the 16-byte boundary below them), scale/zero words and pivot bytes
+  auto issue = [&](uint32_t trel0, uint32_t su, uint8_t *slot) {   // su = unit index inside the segment
+    uint32_t off, len;
+    if (unit_range(trel0, s_pre[su], s_bm[su], off, len)) {
+      const uint64_t g = pay_off0 + off;
+      const uint8_t *src = payload + (g & ~15ull);
+      const uint32_t npieces = ((uint32_t)(g & 15ull) + len + 15u) >> 4;
+#pragma unroll
+      for (int i = 0; i < (S::PAY + 511) / 512; ++i)
+        if ((uint32_t)(i * 32 + lane) < npieces)
+          cp_async16(slot + (size_t)(i * 32 + lane) * 16, src + (size_t)(i * 32 + lane) * 16, 16);
+      const uint64_t t0 = tile_cta + trel0;
+      if (lane < 8) cp_async16(slot + S::PAY + lane * 16, a.packed + a.off_sz + t0 * 4 + lane * 16, 16);
       else if (lane < 10)
-        cp_async16(slot + S::PAY + 128 + (lane - 8) * 16, a.packed + a.off_pivot + u * 32 + (lane - 8) * 16, 16);
+        cp_async16(slot + S::PAY + 128 + (lane - 8) * 16, a.packed + a.off_pivot + t0 + (lane - 8) * 16, 16);
     }
   };
   auto prime = [&](uint64_t s0, uint64_t s1) {
 #pragma unroll
     for (int st = 0; st < NST; ++st) {
       const uint64_t u = s0 + warp + (uint64_t)st * kWarps;
-      if (u < s1) issue(u, (uint32_t)(u - s0), ring + (size_t)st * S::SLOT);
+      if (u < s1) issue((uint32_t)(u - u0) * 32u, (uint32_t)(u - s0), ring + (size_t)st * S::SLOT);
       cp_async_commit();
     }
   };
@@ -990,14 +999,25 @@ __global__ void __launch_bounds__(kThreads, 2) decode_stream_kernel(const Args a
     }
     __syncwarp();
   };
+  // the same for the 32 consecutive tiles of a unit: one base address, constant strides
+  auto copy_out_unit = [&](unsigned rows, uint8_t *dst0) {   // dst0 = first byte of the unit's rows + lane * 16
+    __syncwarp();
+#pragma unroll
+    for (int i = 0; i < C::CPR; ++i) {
+      const int piece = i * 32 + lane, r = piece / C::CPR, q = piece % C::CPR;
+      const uint4 v = *reinterpret_cast<const uint4 *>(ostage + (size_t)phys_chunk<C>(r, q) * 16);
+      if (rows == 0xffffffffu || ((rows >> r) & 1u)) __stcs(reinterpret_cast<uint4 *>(dst0 + (size_t)i * 512), v);
+    }
+    __syncwarp();
+  };
   // the first n (<= 32) held-back tiles, lane j on the j-th
   auto run_flagged = [&](uint32_t n) {
     const uint32_t e = (qhead + lane) & (kQueueCap - 1);
     const uint32_t ft = s_q[warp][0][e], fh = s_q[warp][1][e];
     if ((uint32_t)lane < n) {
-      const uint64_t tile = tile_cta + ft;
-      const uint64_t off = (uint64_t)(C::G / 8) * ((uint64_t)a.lo * tile + base_hi + (fh >> 1));
-      decode_flagged_row<C>(payload + off, a.lo + (fh & 1u), narrow, s_q[warp][2][e], s_q[warp][3][e], ostage, lane);
+      const uint32_t off = (uint32_t)(C::G / 8) * (a.lo * ft + (fh >> 1));
+      decode_flagged_row<C>(payload + pay_off0 + off, a.lo + (fh & 1u), narrow, s_q[warp][2][e], s_q[warp][3][e],
+                            ostage, lane);
     }
     copy_out(n >= 32u ? 0xffffffffu : ((1u << n) - 1u), [&](int r) { return tile_cta + __shfl_sync(kFull, ft, r); });
     qhead = (qhead + n) & (kQueueCap - 1);
@@ -1018,32 +1038,32 @@ __global__ void __launch_bounds__(kThreads, 2) decode_stream_kernel(const Args a
       if (blockIdx.x == gridDim.x - 1 && threadIdx.x == 0 && a.mixed && !stop && base_hi + mine != a.n_groups * a.k_hi)
         atomicOr(a.status, 2u /* TAHQ_DEV_BAD_BITMAP */);
       if (stop) return;
+      pay_off0 = (uint64_t)(C::G / 8) * ((uint64_t)a.lo * tile_cta + base_hi);
     }
     prime(s0, s1);
 
     int slot_i = 0;
-    for (uint64_t u = s0 + warp; u < s1; u += kWarps) {
+    const uint32_t su1 = (uint32_t)(s1 - s0), seg_rel = (uint32_t)(s0 - u0) * 32u;
+    for (uint32_t su = warp; su < su1; su += kWarps) {   // su = unit index inside the segment
       cp_async_wait<NST - 1>();
       __syncwarp();
       if (qn >= 32u) run_flagged(32u);
 
-      const uint32_t su = (uint32_t)(u - s0);
       uint8_t *slot = ring + (size_t)slot_i * S::SLOT;
-      const uint32_t word = s_bm[su];
+      const uint32_t word = s_bm[su], pre = s_pre[su];
       const uint32_t hi = (word >> lane) & 1u;
-      const uint32_t hib = s_pre[su] + (uint32_t)__popc(word & lt);
-      const uint64_t tile = u * 32 + lane;
-      uint64_t off;
-      uint32_t len;
-      const bool fits = unit_range(u, s_pre[su], word, off, len);
-      const bool live = tile < a.n_tiles && fits;
+      const uint32_t hib = pre + (uint32_t)__popc(word & lt);
+      const uint32_t trel0 = seg_rel + su * 32u, trel = trel0 + lane;   // relative to the CTA's first tile
+      uint32_t off, len;
+      const bool fits = unit_range(trel0, pre, word, off, len);
+      const bool live = trel < n_rel && fits;
       const uint32_t szw = reinterpret_cast<const uint32_t *>(slot + S::PAY)[lane];
       const uint32_t pvb = live ? slot[S::PAY + 128 + lane] : 0u;
       const bool flagged = (pvb & 0x80u) != 0;
       const unsigned held = __ballot_sync(kFull, flagged);
       if (flagged) {   // Eq. 4 inverted costs three times the plain path: held back until 32 have gathered
         const uint32_t e = (qhead + qn + (uint32_t)__popc(held & lt)) & (kQueueCap - 1);
-        s_q[warp][0][e] = (uint32_t)(tile - tile_cta);
+        s_q[warp][0][e] = trel;
         s_q[warp][1][e] = (hib << 1) | hi;
         s_q[warp][2][e] = szw;
         s_q[warp][3][e] = pvb;
@@ -1052,7 +1072,7 @@ __global__ void __launch_bounds__(kThreads, 2) decode_stream_kernel(const Args a
       if (live && !flagged) {
         const float s = __half2float(__ushort_as_half((unsigned short)(szw & 0xffffu)));
         const float z = __half2float(__ushort_as_half((unsigned short)(szw >> 16)));
-        const uint8_t *codes = slot + (uint32_t)(off & 15ull) + (uint32_t)(C::G / 8) * (a.lo * lane + (hib - s_pre[su]));
+        const uint8_t *codes = slot + (uint32_t)((pay_off0 + off) & 15ull) + (uint32_t)(C::G / 8) * (a.lo * lane + (hib - pre));
         float x[C::EPT];
         dequant_row<C>(codes, a.lo + hi, narrow, s, z, x);
 #pragma unroll
@@ -1061,12 +1081,13 @@ __global__ void __launch_bounds__(kThreads, 2) decode_stream_kernel(const Args a
       }
       __syncwarp();
       {   // the slot is free again
-        const uint64_t un = u + (uint64_t)NST * kWarps;
-        if (un < s1) issue(un, (uint32_t)(un - s0), slot);
+        const uint32_t sn = su + (uint32_t)NST * kWarps;
+        if (sn < su1) issue(seg_rel + sn * 32u, sn, slot);
         cp_async_commit();
       }
       slot_i = (slot_i + 1 == NST) ? 0 : slot_i + 1;
-      copy_out(__ballot_sync(kFull, live && !flagged), [&](int r) { return u * 32 + (uint64_t)r; });
+      copy_out_unit(__ballot_sync(kFull, live && !flagged),
+                    a.out + (tile_cta + trel0) * (uint64_t)C::ROWB + (size_t)lane * 16);
     }
     cp_async_wait<0>();
     __syncwarp();
