@@ -390,6 +390,9 @@ __device__ __forceinline__ void quant_phase(const Args &a, const void *tmap, uin
   __shared__ uint32_t s_wsum[kWarps];
   __shared__ uint32_t s_qtile[kWarps][kQueueCap];   // held-back tile: (tile - first tile of the CTA) * 2 + higher width
   __shared__ uint32_t s_qhib[kWarps][kQueueCap];    // held-back tile: higher-width tiles before it, from the CTA's first
+  __shared__ uint32_t s_pool[2][kWarps * 32];        // the warps' last, partly filled batches, pooled at the end
+  __shared__ uint32_t s_pool_n;
+  if (threadIdx.x == 0) s_pool_n = 0;   // (read only after barriers further down)
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const unsigned lt = (1u << lane) - 1u;
   UnitRing<C, NST> ring;
@@ -577,13 +580,37 @@ __device__ __forceinline__ void quant_phase(const Args &a, const void *tmap, uin
     __syncwarp();
     seg_hi += seg_total;
   }
-  // ---- what is still held back
+  // ---- what is still held back: full batches first, then the warps pool their remainders so that the
+  // CTA runs as few partly filled batches as possible (on a small tensor these are half of all batches)
   if (f_n) run_flagged();
-  while (qn) {
-    gather(qn < 32u ? qn : 32u);
+  while (qn >= 32u) {
+    gather(32u);
     cp_async_wait<0>();
     __syncwarp();
     run_flagged();
+  }
+  {
+    uint32_t base = 0;
+    if (lane == 0 && qn) base = atomicAdd(&s_pool_n, qn);
+    base = __shfl_sync(kFull, base, 0);
+    if ((uint32_t)lane < qn) {
+      s_pool[0][base + lane] = s_qtile[warp][(qhead + lane) & (kQueueCap - 1)];
+      s_pool[1][base + lane] = s_qhib[warp][(qhead + lane) & (kQueueCap - 1)];
+    }
+    __syncthreads();
+    const uint32_t n = s_pool_n;
+    for (uint32_t t0 = (uint32_t)warp * 32u; t0 < n; t0 += kWarps * 32u) {
+      const uint32_t cnt = n - t0 < 32u ? n - t0 : 32u;
+      s_qtile[warp][lane] = (uint32_t)lane < cnt ? s_pool[0][t0 + lane] : 0u;   // through the warp's own queue
+      s_qhib[warp][lane] = (uint32_t)lane < cnt ? s_pool[1][t0 + lane] : 0u;
+      __syncwarp();
+      qhead = 0;
+      qn = cnt;
+      gather(cnt);
+      cp_async_wait<0>();
+      __syncwarp();
+      run_flagged();
+    }
   }
 }
 
