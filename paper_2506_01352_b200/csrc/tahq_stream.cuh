@@ -182,15 +182,19 @@ __device__ __forceinline__ void stats_phase(const Args &a, const void *tmap, uin
     const uint64_t g_end = (g + 1) * a.tiles_per_group;            // first tile of the next group
     uint64_t ue = (g_end + 31) / 32;
     if (ue > u1 || !use_hist) ue = u1;
+    // The stretch is read back to front: the units read last are the ones the encoder, which walks the same
+    // stretch front to back right afterwards, asks for first, while they are still in L2.
+    const uint64_t nu = ue - us;
 #pragma unroll
     for (int s = 0; s < NST; ++s) {
-      const uint64_t u = us + warp + (uint64_t)s * kWarps;
-      if (u < ue) ring.issue(a, u, s);
+      const uint64_t k = warp + (uint64_t)s * kWarps;
+      if (k < nu) ring.issue(a, ue - 1 - k, s);
       ring.commit();
     }
     __syncthreads();   // the histogram is clear
     int slot = 0;
-    for (uint64_t u = us + warp; u < ue; u += kWarps) {
+    for (uint64_t k = warp; k < nu; k += kWarps) {
+      const uint64_t u = ue - 1 - k;
       ring.wait(a, slot);
       const uint8_t *stage = ring.slot(slot);
       // small groups are ranked on exact scores; large ones are screened first (see select_kernel)
@@ -198,8 +202,8 @@ __device__ __forceinline__ void stats_phase(const Args &a, const void *tmap, uin
                                      : tile_score_screen<C>(stage, lane, a.eps_l1);
       __syncwarp();
       {
-        const uint64_t un = u + (uint64_t)NST * kWarps;
-        if (un < ue) ring.issue(a, un, slot);
+        const uint64_t kn = k + (uint64_t)NST * kWarps;
+        if (kn < nu) ring.issue(a, ue - 1 - kn, slot);
         ring.commit();
       }
       slot = (slot + 1 == NST) ? 0 : slot + 1;
@@ -417,6 +421,7 @@ __device__ __forceinline__ void quant_phase(const Args &a, const void *tmap, uin
       ring.commit();
     }
   };
+
   prime(u0, u0 + kSegWords < u1 ? u0 + kSegWords : u1);
 
   if (blockIdx.x == 0) {   // header and the zero padding behind every section
