@@ -58,6 +58,7 @@ __device__ __forceinline__ float warp_max(float m) {
 // per-tensor mode: max |c g| over the whole tensor (non-negative floats order like their bit patterns)
 template <bool BF16>
 __global__ void __launch_bounds__(kQThreads) qnaive_max_kernel(const QArgs a) {
+  grid_dependency_wait();   // launched as a programmatic dependent of the kernel in front
   const uint64_t n8 = a.tokens * (uint64_t)(a.hidden / 8);
   float m = 0.0f;
   for (uint64_t i = (uint64_t)blockIdx.x * kQThreads + threadIdx.x; i < n8; i += (uint64_t)gridDim.x * kQThreads) {
@@ -72,6 +73,7 @@ __global__ void __launch_bounds__(kQThreads) qnaive_max_kernel(const QArgs a) {
 
 template <bool BF16>
 __global__ void __launch_bounds__(kQThreads, 2) qnaive_encode_kernel(const QArgs a) {
+  grid_dependency_wait();   // launched as a programmatic dependent of the kernel in front
   constexpr int ESZ = BF16 ? 2 : 4;
   const int lane = threadIdx.x & 31;
   const uint64_t warp = ((uint64_t)blockIdx.x * kQThreads + threadIdx.x) >> 5;
@@ -246,6 +248,7 @@ __global__ void __launch_bounds__(kQThreads, 2) qnaive_encode_kernel(const QArgs
 
 template <bool BF16>
 __global__ void __launch_bounds__(kQThreads) qnaive_decode_kernel(const QArgs a) {
+  grid_dependency_wait();   // launched as a programmatic dependent of the kernel in front
   constexpr int ESZ = BF16 ? 2 : 4;
   const int lane = threadIdx.x & 31;
   const uint64_t warp = ((uint64_t)blockIdx.x * kQThreads + threadIdx.x) >> 5;

@@ -2,9 +2,11 @@
 // buffer and of the workspace, kernel selection and launches on the caller's stream.
 #include "../../include/tahq.h"
 
+#include <algorithm>
 #include <atomic>
 #include <cstdlib>
 #include <cstring>
+#include <utility>
 #include <vector>
 
 #include "tahq_stream.cuh"
@@ -216,6 +218,34 @@ static int prepare(K kernel, int smem, const DevInfo &d, std::atomic<int> *cache
   return occ;
 }
 
+// Launch a kernel as a programmatic dependent of the kernel in front of it in the stream: the launch is set up
+// while that kernel still runs (about 2 us less per kernel boundary, measured); the kernel starts with
+// griddepcontrol.wait, so it reads nothing before that kernel is done.
+template <class... P, class... A>
+static cudaError_t launch_dependent(void (*kernel)(P...), unsigned grid, unsigned block, size_t smem, cudaStream_t st,
+                                    A &&...args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(block);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, std::forward<A>(args)...);
+}
+
+// Zero the first `bytes` (a multiple of 16) of the workspace with a kernel, so that the call's next kernel can
+// be its programmatic dependent.
+static tahq_status clear_workspace(void *d_ws, uint64_t bytes, cudaStream_t st) {
+  const uint64_t n16 = bytes / 16;
+  const unsigned grid = (unsigned)std::min<uint64_t>((n16 + kThreads - 1) / kThreads, 592);
+  TAHQ_LAUNCH("clear", st, clear_kernel<<<grid ? grid : 1, kThreads, 0, st>>>(static_cast<uint4 *>(d_ws), n16));
+  return cudaGetLastError() == cudaSuccess ? TAHQ_OK : TAHQ_ERR_CUDA;
+}
+
 template <class C> struct Stages {
   static constexpr int STATS = 2;
   static constexpr int QUANT = (C::ROWB == 256) ? 2 : (C::ROWB == 128 ? 2 : 3);
@@ -294,8 +324,7 @@ static tahq_status encode_t(const Plan &pl, const Args &a_in, cudaStream_t st) {
     const uint64_t n_alloc = a.n_tiles / pl.alloc_m;
     const uint64_t want = (n_alloc + kWarps - 1) / kWarps, cap = (uint64_t)d.sms * 8;
     const unsigned grid = (unsigned)(want < cap ? want : cap);
-    if (C::BF16) TAHQ_LAUNCH("alloc_score", st, alloc_score_kernel<true><<<grid, kThreads, 0, st>>>(a));
-    else TAHQ_LAUNCH("alloc_score", st, alloc_score_kernel<false><<<grid, kThreads, 0, st>>>(a));
+    TAHQ_LAUNCH("alloc_score", st, launch_dependent(alloc_score_kernel<C::BF16>, grid, kThreads, 0, st, a));
   }
   if (pl.mixed) {
     if (pl.alloc_m > 1) {
@@ -307,14 +336,15 @@ static tahq_status encode_t(const Plan &pl, const Args &a_in, cudaStream_t st) {
       if (!occ) return TAHQ_ERR_CUDA;
       const uint64_t n_units = (a.n_tiles + 31) / 32;
       TAHQ_LAUNCH("stats", st,
-                  stats_stream_kernel<C, NS><<<persistent_grid((n_units + kWarps - 1) / kWarps, d, occ), kThreads, smem,
-                                               st>>>(a, tmap));
+                  launch_dependent(stats_stream_kernel<C, NS>, persistent_grid((n_units + kWarps - 1) / kWarps, d, occ),
+                                   kThreads, smem, st, a, tmap));
     } else {
       constexpr int NS = Stages<C>::STATS;
       const int smem = NS * C::STAGE_BYTES;
       const int occ = prepare(stats_kernel<C, NS>, smem, d, occ_stats);
       if (!occ) return TAHQ_ERR_CUDA;
-      TAHQ_LAUNCH("stats", st, stats_kernel<C, NS><<<persistent_grid(n_chunks, d, occ), kThreads, smem, st>>>(a));
+      TAHQ_LAUNCH("stats", st,
+                  launch_dependent(stats_kernel<C, NS>, persistent_grid(n_chunks, d, occ), kThreads, smem, st, a));
     }
     const int sel_smem = kSortCap * 8;
     if (!sel_ready[d.dev & 63].load(std::memory_order_acquire)) {
@@ -322,7 +352,8 @@ static tahq_status encode_t(const Plan &pl, const Args &a_in, cudaStream_t st) {
         return TAHQ_ERR_CUDA;
       sel_ready[d.dev & 63].store(1, std::memory_order_release);
     }
-    TAHQ_LAUNCH("select", st, select_kernel<<<(unsigned)(a.n_groups * a.cpg), kSelThreads, sel_smem, st>>>(a));
+    TAHQ_LAUNCH("select", st,
+                launch_dependent(select_kernel, (unsigned)(a.n_groups * a.cpg), kSelThreads, sel_smem, st, a));
   }
   if constexpr (C::LPT == 1) {   // one lane per tile: warps stream units of 32 tiles independently
     constexpr int NQ = 2;
@@ -330,16 +361,15 @@ static tahq_status encode_t(const Plan &pl, const Args &a_in, cudaStream_t st) {
     const int occ = prepare(quant_pack_stream_kernel<C, NQ, SR>, smem, d, occ_quant);
     if (!occ) return TAHQ_ERR_CUDA;
     const uint64_t n_units = (a.n_tiles + 31) / 32;
-    TAHQ_LAUNCH("quant_pack", st,
-                quant_pack_stream_kernel<C, NQ, SR><<<persistent_grid((n_units + kWarps - 1) / kWarps, d, occ), kThreads,
-                                                  smem, st>>>(a, tmap));
+    const unsigned grid = persistent_grid((n_units + kWarps - 1) / kWarps, d, occ);
+    TAHQ_LAUNCH("quant_pack", st, launch_dependent(quant_pack_stream_kernel<C, NQ, SR>, grid, kThreads, smem, st, a, tmap));
   } else {
     constexpr int NQ = Stages<C>::QUANT;
     const int smem = NQ * (C::STAGE_BYTES + C::TPC * 4);
     const int occ = prepare(quant_pack_kernel<C, NQ, SR>, smem, d, occ_quant);
     if (!occ) return TAHQ_ERR_CUDA;
     TAHQ_LAUNCH("quant_pack", st,
-                quant_pack_kernel<C, NQ, SR><<<persistent_grid(n_chunks, d, occ), kThreads, smem, st>>>(a));
+                launch_dependent(quant_pack_kernel<C, NQ, SR>, persistent_grid(n_chunks, d, occ), kThreads, smem, st, a));
   }
   return cudaGetLastError() == cudaSuccess ? TAHQ_OK : TAHQ_ERR_CUDA;
 }
@@ -357,8 +387,8 @@ static tahq_status decode_t(const Plan &pl, const Args &a, cudaStream_t st) {
     if (!occ) return TAHQ_ERR_CUDA;
     const uint64_t n_units = (a.n_tiles + 31) / 32;
     TAHQ_LAUNCH("decode", st,
-                decode_stream_kernel<C><<<persistent_grid((n_units + kWarps - 1) / kWarps, d, occ), kThreads, smem,
-                                          st>>>(a));
+                launch_dependent(decode_stream_kernel<C>, persistent_grid((n_units + kWarps - 1) / kWarps, d, occ),
+                                 kThreads, smem, st, a));
   } else {
     const int smem = DecSmem<C>::TOTAL;
     const int occ = prepare(decode_kernel<C>, smem, d, occ_dec);
@@ -366,7 +396,7 @@ static tahq_status decode_t(const Plan &pl, const Args &a, cudaStream_t st) {
     unsigned grid = persistent_grid(n_chunks, d, occ);
     const uint64_t need = (n_chunks + kChunkCap - 1) / kChunkCap;   // a CTA keeps its chunks' bit map in shared memory
     if (grid < need) grid = (unsigned)need;
-    TAHQ_LAUNCH("decode", st, decode_kernel<C><<<grid, kThreads, smem, st>>>(a));
+    TAHQ_LAUNCH("decode", st, launch_dependent(decode_kernel<C>, grid, kThreads, smem, st, a));
   }
   return cudaGetLastError() == cudaSuccess ? TAHQ_OK : TAHQ_ERR_CUDA;
 }
@@ -418,7 +448,7 @@ tahq_status tahq_encode(const tahq_params *p, const void *d_in, void *d_packed, 
   fill_args(p, pl, static_cast<uint8_t *>(d_ws), &a);
   a.in = static_cast<const uint8_t *>(d_in);
   a.packed = static_cast<uint8_t *>(d_packed);
-  if (cudaMemsetAsync(d_ws, 0, pl.ws_zero_end, st) != cudaSuccess) return TAHQ_ERR_CUDA;
+  if (clear_workspace(d_ws, pl.ws_zero_end, st) != TAHQ_OK) return TAHQ_ERR_CUDA;
   const bool bf = p->dtype == TAHQ_BF16;
   if (p->rounding == 1) {   // stochastic rounding: kernels of their own, the default path carries none of it
     switch (p->tile) {
@@ -452,7 +482,7 @@ tahq_status tahq_decode(const tahq_params *p, const void *d_packed, size_t packe
   fill_args(p, pl, static_cast<uint8_t *>(d_ws), &a);
   a.packed = const_cast<uint8_t *>(static_cast<const uint8_t *>(d_packed));
   a.out = static_cast<uint8_t *>(d_out);
-  if (cudaMemsetAsync(d_ws, 0, pl.ws_ncand, st) != cudaSuccess) return TAHQ_ERR_CUDA;   // status + flags
+  if (clear_workspace(d_ws, pl.ws_ncand, st) != TAHQ_OK) return TAHQ_ERR_CUDA;   // status + flags
   const bool bf = p->dtype == TAHQ_BF16;
   switch (p->tile) {
     case 8: return bf ? decode_t<Cfg<8, true>>(pl, a, st) : decode_t<Cfg<8, false>>(pl, a, st);
@@ -546,14 +576,14 @@ tahq_status tahq_qnaive_encode(const tahq_qnaive_params *p, const void *d_in, vo
   q_args(p, q, &a, d_ws);
   a.in = static_cast<const uint8_t *>(d_in);
   a.packed = static_cast<uint8_t *>(d_packed);
-  if (cudaMemsetAsync(d_ws, 0, 256, st) != cudaSuccess) return TAHQ_ERR_CUDA;
+  if (clear_workspace(d_ws, 256, st) != TAHQ_OK) return TAHQ_ERR_CUDA;
   const bool bf = p->dtype == TAHQ_BF16;
   if (p->per_tensor) {
-    if (bf) TAHQ_LAUNCH("qnaive_max", st, qnaive_max_kernel<true><<<d.sms * 4, kQThreads, 0, st>>>(a));
-    else TAHQ_LAUNCH("qnaive_max", st, qnaive_max_kernel<false><<<d.sms * 4, kQThreads, 0, st>>>(a));
+    if (bf) TAHQ_LAUNCH("qnaive_max", st, launch_dependent(qnaive_max_kernel<true>, d.sms * 4, kQThreads, 0, st, a));
+    else TAHQ_LAUNCH("qnaive_max", st, launch_dependent(qnaive_max_kernel<false>, d.sms * 4, kQThreads, 0, st, a));
   }
-  if (bf) TAHQ_LAUNCH("qnaive_encode", st, qnaive_encode_kernel<true><<<q_grid(p->tokens, d), kQThreads, 0, st>>>(a));
-  else TAHQ_LAUNCH("qnaive_encode", st, qnaive_encode_kernel<false><<<q_grid(p->tokens, d), kQThreads, 0, st>>>(a));
+  if (bf) TAHQ_LAUNCH("qnaive_encode", st, launch_dependent(qnaive_encode_kernel<true>, q_grid(p->tokens, d), kQThreads, 0, st, a));
+  else TAHQ_LAUNCH("qnaive_encode", st, launch_dependent(qnaive_encode_kernel<false>, q_grid(p->tokens, d), kQThreads, 0, st, a));
   return cudaGetLastError() == cudaSuccess ? TAHQ_OK : TAHQ_ERR_CUDA;
 }
 
@@ -572,11 +602,11 @@ tahq_status tahq_qnaive_decode(const tahq_qnaive_params *p, const void *d_packed
   q_args(p, q, &a, d_ws);
   a.packed = const_cast<uint8_t *>(static_cast<const uint8_t *>(d_packed));
   a.out = static_cast<uint8_t *>(d_out);
-  if (cudaMemsetAsync(d_ws, 0, 256, st) != cudaSuccess) return TAHQ_ERR_CUDA;
+  if (clear_workspace(d_ws, 256, st) != TAHQ_OK) return TAHQ_ERR_CUDA;
   if (p->dtype == TAHQ_BF16)
-    TAHQ_LAUNCH("qnaive_decode", st, qnaive_decode_kernel<true><<<q_grid(p->tokens, d), kQThreads, 0, st>>>(a));
+    TAHQ_LAUNCH("qnaive_decode", st, launch_dependent(qnaive_decode_kernel<true>, q_grid(p->tokens, d), kQThreads, 0, st, a));
   else
-    TAHQ_LAUNCH("qnaive_decode", st, qnaive_decode_kernel<false><<<q_grid(p->tokens, d), kQThreads, 0, st>>>(a));
+    TAHQ_LAUNCH("qnaive_decode", st, launch_dependent(qnaive_decode_kernel<false>, q_grid(p->tokens, d), kQThreads, 0, st, a));
   return cudaGetLastError() == cudaSuccess ? TAHQ_OK : TAHQ_ERR_CUDA;
 }
 

@@ -58,6 +58,12 @@ __device__ __forceinline__ void cp_async16(void *smem, const void *gmem, int src
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(s), "l"(gmem), "r"(src_bytes)
                : "memory");
 }
+// Programmatic dependent launch: a kernel launched with the stream-serialisation attribute is set up while the
+// kernel in front of it in the stream still runs; it must call this before it touches anything that kernel
+// writes (it returns once that whole grid is done and its writes are visible).  A no-op in a kernel launched
+// the ordinary way.  No kernel here signals its dependents early: measured, that only made things slower.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void cp_async_wait() {

@@ -140,6 +140,13 @@ __device__ __forceinline__ uint64_t cta_exclusive_prefix(const Args &a, uint64_t
 
 // Self-test of the bounded waits: CTA 1 waits for a count that CTA 0 never publishes.  The wait gives
 // up after kSpinLimit polls, the status word gets TAHQ_DEV_TIMEOUT, and the kernel returns.
+// Clears the part of the workspace that a call needs zeroed (status word, look-back flags, counters,
+// histograms); the call's first tile kernel is launched as its programmatic dependent.
+__global__ void __launch_bounds__(kThreads) clear_kernel(uint4 *p, uint64_t n16) {
+  for (uint64_t i = blockIdx.x * (uint64_t)kThreads + threadIdx.x; i < n16; i += (uint64_t)gridDim.x * kThreads)
+    p[i] = make_uint4(0, 0, 0, 0);
+}
+
 __global__ void __launch_bounds__(kThreads) wait_selftest_kernel(const Args a) {
   if (blockIdx.x == 0) return;
   bool unused;
@@ -154,6 +161,7 @@ __global__ void __launch_bounds__(kThreads, 2) stats_kernel(const Args a) {
   extern __shared__ __align__(128) uint8_t smem[];
   __shared__ uint32_t s_hist[kBins];
   const bool use_hist = !a.direct;
+  grid_dependency_wait();
   if (use_hist) {
     for (int b = threadIdx.x; b < kBins; b += kThreads) s_hist[b] = 0;
     __syncthreads();
@@ -250,6 +258,7 @@ __global__ void __launch_bounds__(kThreads) alloc_score_kernel(const Args a) {
   const uint64_t n_warps = ((uint64_t)gridDim.x * kThreads) >> 5;
   const uint32_t A = a.alloc_m * a.tile, n_oct = A / 8;
   const uint64_t n_alloc = a.n_tiles / a.alloc_m;
+  grid_dependency_wait();
   for (uint64_t t = warp; t < n_alloc; t += n_warps) {
     const uint8_t *base = a.in + t * (uint64_t)A * (BF16 ? 2 : 4);
     const float L1 = alloc_tree<BF16>(base, n_oct, lane, [](float m) { return m; });
@@ -354,6 +363,7 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const Args a) {
   const float *sc = a.scores + g * ng;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   auto from_smem = [&](uint64_t i, unsigned long long &key) { key = s_keys[i]; return true; };
+  grid_dependency_wait();   // scores and histograms are the score kernel's
 
   if (a.direct) {   // small group: rank all of its tiles here (one CTA per group)
     for (uint32_t i = threadIdx.x; i < (uint32_t)ng; i += kSelThreads) s_keys[i] = rank_key(sc[i], i);
@@ -848,6 +858,7 @@ template <class C, int NST, bool SR>
 __global__ void __launch_bounds__(kThreads, 2) quant_pack_kernel(const Args a) {
   extern __shared__ __align__(128) uint8_t smem[];
   static_assert(C::LPT == 2, "tiles owned by one lane go through quant_pack_stream_kernel");
+  grid_dependency_wait();
   __shared__ uint2 s_cnt[kThreads / 32];
   uint32_t *sz32 = reinterpret_cast<uint32_t *>(a.packed + a.off_sz);
   uint8_t *pivot = a.packed + a.off_pivot;
@@ -1053,6 +1064,7 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const Args a) {
   __shared__ uint32_t s_bm[kBmCap];         // bit map of this CTA's tiles (tail bits cleared)
   __shared__ uint16_t s_chi[kChunkCap];     // higher-width tiles per chunk
   static_assert(C::LPT == 2, "tiles owned by one lane go through decode_stream_kernel");
+  grid_dependency_wait();
   __shared__ uint2 s_cnt[kThreads / 32];
   __shared__ uint32_t s_bad;
   const uint32_t *bitmap = reinterpret_cast<const uint32_t *>(a.packed + a.off_bitmap);

@@ -234,6 +234,7 @@ __global__ void __launch_bounds__(kThreads, 2) stats_stream_kernel(const Args a,
   extern __shared__ __align__(1024) uint8_t smem_1k[];
   uint8_t *smem = smem_1k;
   __shared__ uint32_t s_hist[kBins];   // this CTA's counts for the ranking group it is in
+  grid_dependency_wait();   // the histograms are cleared by the kernel in front
   stats_phase<C, NST>(a, &tmap, smem, reinterpret_cast<unsigned long long *>(smem + (size_t)kWarps * NST * StreamCfg<C>::UNIT_BYTES),
                       s_hist);
 }
@@ -623,6 +624,7 @@ template <class C, int NST, bool SR>
 __global__ void __launch_bounds__(kThreads, 2) quant_pack_stream_kernel(const Args a, const __grid_constant__ CUtensorMap tmap) {
   extern __shared__ __align__(1024) uint8_t smem_1k[];
   uint8_t *smem = smem_1k;
+  grid_dependency_wait();   // scores and thresholds are the selection kernel's
   quant_phase<C, NST, SR, false>(a, &tmap, smem);
 }
 
@@ -934,6 +936,7 @@ __global__ void __launch_bounds__(kThreads, 2) decode_stream_kernel(const Args a
                                                    // before it (and the width bit), scale/zero word, pivot byte
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const unsigned lt = (1u << lane) - 1u;
+  grid_dependency_wait();   // the look-back flags are cleared by the kernel in front
   uint8_t *ring = smem + (size_t)warp * S::WARP;
   uint8_t *ostage = ring + (size_t)NST * S::SLOT;
   const uint32_t *bitmap = reinterpret_cast<const uint32_t *>(a.packed + a.off_bitmap);
