@@ -304,6 +304,33 @@ def test_deterministic_and_stream_ordered():
     assert rel < 0.05
 
 
+def test_captured_in_a_cuda_graph_replays_to_the_same_bytes():
+    """Every kernel of a call is a programmatic dependent of the one in front; captured into a CUDA graph
+    the replay writes the oracle's bytes."""
+    x = synth.make("c2_gpt2s", device="cuda")
+    p = T.params_for(x, group_tokens=1024, tile=64, budget_millibits=3800)
+    s = torch.cuda.Stream()
+    ws = T.alloc_workspace(p)
+    pk = T.alloc_packed(p)
+    out = torch.empty_like(x)
+    with torch.cuda.stream(s):
+        T.encode(p, x, packed=pk, ws=ws, stream=s)      # first use outside the capture (one-time attributes)
+        T.decode(p, pk, out=out, ws=ws, stream=s)
+        s.synchronize()
+        pk.fill_(0xA5)
+        out.fill_(float("nan"))
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=s):
+            T.encode(p, x, packed=pk, ws=ws, stream=s)
+            T.decode(p, pk, out=out, ws=ws, stream=s)
+        g.replay()
+        s.synchronize()
+    assert T.device_status(ws) == 0
+    want = O.encode(oparams(p), synth.to_host_array(x))
+    assert np.array_equal(pk.cpu().numpy(), want)
+    assert np.array_equal(synth.to_host_array(out).view(np.uint32), O.decode(oparams(p), want).view(np.uint32))
+
+
 def test_bounded_wait_runs_out_and_reports():
     """A device-side wait on a flag that nothing sets gives up after its fixed number of polls: the kernel
     returns, the status word says TIMEOUT, and the context goes on working (an encode right after it)."""
