@@ -45,7 +45,7 @@ struct Plan {
   uint32_t f;             // budget % 1000
   bool mixed;             // two widths in use (k_hi > 0)
   bool direct;            // small ranking groups: select straight from the scores
-  uint32_t cpg, cand_cap;
+  uint32_t cpg, cand_cap, sel_m;
   uint32_t alloc_m;            // quantisation tiles per allocation tile (Sec. 3.2; 1 by default)
   uint64_t rank_per_group, rank_k;   // allocation tiles per ranking group, and how many of them get the higher width
   // workspace offsets
@@ -108,9 +108,15 @@ static tahq_status make_plan(const tahq_params *p, Plan *pl) {
   pl->mixed = L.k_hi > 0;
   pl->direct = pl->rank_per_group <= (uint64_t)kSortCap;
   pl->cpg = 1;
+  pl->sel_m = 1;
   pl->cand_cap = 0;
   if (pl->mixed && !pl->direct) {
-    pl->cpg = (uint32_t)((pl->rank_per_group + kSelSlice - 1) / kSelSlice);
+    // one CTA per slice of the group's scores, or several slices per CTA so that the grid stays near one wave
+    const uint64_t slices = (pl->rank_per_group + kSelSlice - 1) / kSelSlice;
+    uint64_t m = (slices * L.n_groups + 255) / 256;
+    m = m < 1 ? 1 : m > 64 ? 64 : m;
+    pl->sel_m = (uint32_t)m;
+    pl->cpg = (uint32_t)((slices + m - 1) / m);
     // select_kernel copes with more candidates than the list holds; the single-launch encode does not, so
     // there the list holds a whole group (every tile is a candidate when all scores are equal)
     const uint64_t cap = fused_encode_wanted() ? 0xffffffffull : 32768ull;
@@ -191,6 +197,7 @@ static void fill_args(const tahq_params *p, const Plan &pl, uint8_t *ws, Args *a
   a->cand = reinterpret_cast<unsigned long long *>(ws + pl.ws_cand);
   a->cand_cap = pl.cand_cap;
   a->cpg = pl.cpg;
+  a->sel_m = pl.sel_m;
   a->direct = pl.direct;
   // the screening score leaves varsigma out; its share of the score is below G * varsigma / ln 2
   a->exact_scores = pl.direct || pl.alloc_m > 1 || (double)p->tile * (double)p->eps_log > 1e-5;

@@ -37,6 +37,7 @@ struct Args {
   unsigned long long *theta;// [n_groups] ranking key of the k_hi-th ranked tile
   unsigned long long *cand; // [n_groups][cand_cap]
   uint32_t cand_cap, cpg;   // candidate capacity per group; CTAs per group of select_kernel
+  uint32_t sel_m;           // slices of kSelSlice scores that one CTA of select_kernel takes
   uint32_t direct;          // small groups: select_kernel ranks all scores of the group itself
   uint32_t exact_scores;    // stats_kernel writes exact scores (small groups, or a varsigma too large to screen)
   unsigned long long *flags;// [kMaxGrid] (zeroed per call) per-CTA published counts for the offset prefix
@@ -373,12 +374,12 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const Args a) {
     return;
   }
 
-  // this CTA's slice of the group's scores, in flight while the threshold bin is being found
-  const uint64_t lo = (blockIdx.x % a.cpg) * (uint64_t)kSelSlice;
+  // this CTA's first slice of the group's scores, in flight while the threshold bin is being found
+  const uint64_t lo0 = (blockIdx.x % a.cpg) * (uint64_t)a.sel_m * kSelSlice;
   float sv[4];
 #pragma unroll
   for (int u = 0; u < 4; ++u) {
-    const uint64_t i = lo + (uint64_t)u * kSelThreads + threadIdx.x;
+    const uint64_t i = lo0 + (uint64_t)u * kSelThreads + threadIdx.x;
     sv[u] = i < ng ? __ldg(sc + i) : 0.0f;
   }
 
@@ -414,48 +415,30 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const Args a) {
   // is more than 2*kScreenErr above (below) the bin are certainly inside (outside) the top k_hi: their
   // score is replaced by +inf (-inf).  The rest are candidates: their exact score is recomputed from
   // the tensor, stored, and ranked exactly in step C.
-  __shared__ uint32_t s_list[kSelSlice];
-  __shared__ uint32_t s_nlist, s_nabove;
+  // A CTA takes sel_m consecutive slices (a large tensor still fills the GPU only once, so the chain of
+  // dependent steps above and below is paid once, not once per wave of CTAs).  Candidates collect in the
+  // shared memory that step C uses for its keys; they are re-scored when the next slice might not fit,
+  // and at the end.
+  uint32_t *s_list = reinterpret_cast<uint32_t *>(s_keys);   // index inside the group
+  constexpr uint32_t kListCap = 2 * kSortCap;
+  __shared__ uint32_t s_nlist, s_nabove, s_slot0;
   if (threadIdx.x == 0) { s_nlist = 0; s_nabove = 0; }
   __syncthreads();
   float *scw = a.scores + g * ng;
   const float band_lo = (float)B - kScreenBand, band_hi = (float)(B + 1) + kScreenBand;
-#pragma unroll
-  for (int u = 0; u < 4; ++u) {
-    const uint64_t i = lo + (uint64_t)u * kSelThreads + threadIdx.x;
-    const float t = fmaxf(sv[u], 0.0f) * kBinScale;
-    const bool in = i < ng;
-    const bool above = in && t > band_hi, below = in && t < band_lo;
-    if (above) scw[i] = __int_as_float(0x7f800000);
-    if (below) scw[i] = __int_as_float(0xff800000);
-    const unsigned ma = __ballot_sync(kFull, above);
-    if (ma && lane == 0) atomicAdd(&s_nabove, (uint32_t)__popc(ma));
-    const bool take = in && !above && !below;
-    const unsigned m = __ballot_sync(kFull, take);
-    if (m) {
-      uint32_t base = 0;
-      if (lane == 0) base = atomicAdd(&s_nlist, (uint32_t)__popc(m));
-      base = __shfl_sync(kFull, base, 0);
-      if (take) s_list[base + __popc(m & ((1u << lane) - 1u))] = (uint32_t)(i - lo);
-    }
-  }
-  __syncthreads();
-  if (threadIdx.x == 0 && s_nabove) atomicAdd(&a.nabove[g], s_nabove);
-  {
+  const uint32_t tile_bytes = a.tile * (a.bf16 ? 2u : 4u);
+  const uint32_t noct = a.tile / 8, per_round = kSelThreads / noct;
+  const uint32_t sub = threadIdx.x % noct;
+  auto rescore = [&]() {   // called by the whole CTA, after a barrier: s_nlist is settled
     const uint32_t nl = s_nlist;
-    const uint32_t tile_bytes = a.tile * (a.bf16 ? 2u : 4u);
-    uint32_t slot0 = 0;
-    __shared__ uint32_t s_slot0;
     if (threadIdx.x == 0) s_slot0 = atomicAdd(&a.ncand[g], nl);
     __syncthreads();
-    slot0 = s_slot0;
+    const uint32_t slot0 = s_slot0;
     // candidates, densely over the threads: NOCT = tile/8 neighbouring lanes share one candidate
-    const uint32_t noct = a.tile / 8, per_round = kSelThreads / noct;
-    const uint32_t sub = threadIdx.x % noct;
     for (uint32_t j0 = 0; j0 < nl; j0 += per_round) {   // uniform trip count: whole warps take part
       const uint32_t j = j0 + threadIdx.x / noct;
       const bool live = j < nl;
-      const uint64_t i = lo + s_list[live ? j : 0];
+      const uint64_t i = s_list[live ? j : 0];
       const uint8_t *tp = a.in + (g * ng + i) * (uint64_t)tile_bytes;
       float ex;
       if (a.exact_scores) {   // nothing to recompute (and with wider allocation tiles tp is not the tile)
@@ -478,7 +461,51 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const Args a) {
         if (slot0 + j < a.cand_cap) a.cand[g * a.cand_cap + slot0 + j] = rank_key(ex, (uint32_t)i);
       }
     }
+    __syncthreads();
+    if (threadIdx.x == 0) s_nlist = 0;
+    __syncthreads();
+  };
+  uint32_t nl_seen = 0;
+  for (uint32_t m = 0; m < a.sel_m; ++m) {
+    const uint64_t lo = lo0 + (uint64_t)m * kSelSlice;
+    if (lo >= ng) break;
+    float nx[4];   // the next slice's scores, in flight while this one is classified
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const uint64_t i = lo + kSelSlice + (uint64_t)u * kSelThreads + threadIdx.x;
+      nx[u] = (m + 1 < a.sel_m && i < ng) ? __ldg(sc + i) : 0.0f;
+    }
+    if (nl_seen + (uint32_t)kSelSlice > kListCap) {   // (the same value in every thread)
+      rescore();
+      nl_seen = 0;
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const uint64_t i = lo + (uint64_t)u * kSelThreads + threadIdx.x;
+      const float t = fmaxf(sv[u], 0.0f) * kBinScale;
+      const bool in = i < ng;
+      const bool above = in && t > band_hi, below = in && t < band_lo;
+      if (above) scw[i] = __int_as_float(0x7f800000);
+      if (below) scw[i] = __int_as_float(0xff800000);
+      const unsigned ma = __ballot_sync(kFull, above);
+      if (ma && lane == 0) atomicAdd(&s_nabove, (uint32_t)__popc(ma));
+      const bool take = in && !above && !below;
+      const unsigned mk = __ballot_sync(kFull, take);
+      if (mk) {
+        uint32_t base = 0;
+        if (lane == 0) base = atomicAdd(&s_nlist, (uint32_t)__popc(mk));
+        base = __shfl_sync(kFull, base, 0);
+        if (take) s_list[base + __popc(mk & ((1u << lane) - 1u))] = (uint32_t)i;
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) sv[u] = nx[u];
+    __syncthreads();       // the slice's candidates are all listed ...
+    nl_seen = s_nlist;
+    __syncthreads();       // ... and counted by everyone before the next slice adds to them
   }
+  if (threadIdx.x == 0 && s_nabove) atomicAdd(&a.nabove[g], s_nabove);
+  rescore();
 
   // ---- C: the CTA that finishes the group last ranks the candidates exactly
   __threadfence();
