@@ -88,8 +88,8 @@ typedef struct {
                                 hidden and is at most 8192; 0 = tile (the paper's default).  The entropy
                                 is taken over A channels, the top-p% of the S*hidden/A allocation tiles of
                                 a ranking group get the higher width, and every quantisation tile inside
-                                shares it; A = hidden is token-level allocation.  A != tile needs tile 32
-                                or 64 (TAHQ_ERR_UNSUPPORTED otherwise).                              */
+                                shares it; A = hidden is token-level allocation.  A above 8192 is
+                                TAHQ_ERR_UNSUPPORTED.                                                */
 } tahq_params;
 
 /* Byte offsets of the sections of the packed buffer (all multiples of 128). */

@@ -103,7 +103,7 @@ static tahq_status make_plan(const tahq_params *p, Plan *pl) {
   L.off_pivot = up(L.off_scale_zero + 4 * L.n_tiles, 128);
   L.off_payload = up(L.off_pivot + L.n_tiles, 128);
   L.total_bytes = up(L.off_payload + L.payload_bytes, 128);
-  if (pl->alloc_m > 1 && (G == 128 || A > 8192)) return TAHQ_ERR_UNSUPPORTED;
+  if (pl->alloc_m > 1 && A > 8192) return TAHQ_ERR_UNSUPPORTED;
 
   pl->mixed = L.k_hi > 0;
   pl->direct = pl->rank_per_group <= (uint64_t)kSortCap;

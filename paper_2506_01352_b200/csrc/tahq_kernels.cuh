@@ -928,7 +928,10 @@ __global__ void __launch_bounds__(kThreads, 2) quant_pack_kernel(const Args a) {
     const uint32_t nvalid = left < (uint64_t)C::TPC ? (uint32_t)left : (uint32_t)C::TPC;
     const uint32_t own = threadIdx.x / C::LPT;   // tile of the chunk this thread looks at first
     const float *sc_stage = reinterpret_cast<const float *>(stage + C::STAGE_BYTES);   // staged with the rows
-    const bool hi1 = a.mixed && own < nvalid && cur.is_hi_score(a, sc_stage[own], own);
+    // (scores ride along with the rows only when there is one per tile: with wider allocation tiles, Sec. 3.2,
+    // the few scores are read where they lie)
+    const bool hi1 = a.mixed && own < nvalid &&
+                     (a.alloc_m > 1 ? cur.is_hi(a, tile0 + own, own) : cur.is_hi_score(a, sc_stage[own], own));
     const uint64_t goff = (uint64_t)(C::G / 8) * ((uint64_t)a.lo * tile0 + hi_run);
 
     {
@@ -1015,7 +1018,7 @@ __global__ void __launch_bounds__(kThreads, 2) quant_pack_kernel(const Args a) {
       }
     }
     cur.advance(a, C::TPC);
-  }, a.mixed ? a.scores : nullptr);
+  }, (a.mixed && a.alloc_m == 1) ? a.scores : nullptr);
 }
 
 // ------------------------------------------------------------------------------------------

@@ -240,7 +240,8 @@ def test_fused_cooperative_encode_matches_too():
 @pytest.mark.parametrize("name,S,G,A", [("c1_tiny", 64, 64, 128), ("c1_tiny", 64, 64, 256), ("c1_tiny", 64, 32, 128),
                                         ("c2_gpt2s", 1024, 64, 192), ("c2_gpt2s", 1024, 64, 768),
                                         ("c3_llama7b", 2048, 64, 256), ("c3_llama7b", 2048, 64, 4096),
-                                        ("c3_llama7b", 2048, 32, 2048)])
+                                        ("c3_llama7b", 2048, 32, 2048), ("c1_tiny", 64, 128, 256),
+                                        ("c2_gpt2s", 1024, 128, 384), ("c3_llama7b", 2048, 128, 1024)])
 def test_allocation_tile_wider_than_quantisation_tile(name, S, G, A):
     """A = m*G (Sec. 3.2): entropy over A channels, top-p% of the allocation tiles per sample, one width per
     allocation tile; A = hidden is token-level allocation.  Small and large ranking groups, m a power of two or not."""
@@ -254,7 +255,7 @@ def test_allocation_tile_wider_than_quantisation_tile(name, S, G, A):
 def test_allocation_tile_limits():
     x = synth.make("c1_tiny", device="cuda")
     assert T.packed_bound(T.params_for(x, group_tokens=64, tile=64, alloc_tile=96)) == 0          # not a multiple of the tile
-    assert T.packed_bound(T.params_for(x, group_tokens=64, tile=128, alloc_tile=256)) == 0        # 128-wide tiles: not built
+    assert T.packed_bound(T.params_for(x, group_tokens=64, tile=128, alloc_tile=16384)) == 0      # wider than 8192 channels
     assert T.packed_bound(T.params_for(x, group_tokens=64, tile=64, alloc_tile=64)) == \
         T.packed_bound(T.params_for(x, group_tokens=64, tile=64))
 
