@@ -54,7 +54,7 @@ def test_invalid_and_unsupported_parameters():
     base = dict(tokens=128, hidden=256, group_tokens=64, tile=64, budget_millibits=3800)
     for kw in [dict(tile=48), dict(hidden=100), dict(group_tokens=5), dict(budget_millibits=1999),
                dict(budget_millibits=8001), dict(tile=256), dict(dtype=2), dict(tokens=0), dict(tau=-1.0),
-               dict(tile=4), dict(rounding=2), dict(alloc_tile=96), dict(tile=128, alloc_tile=256)]:
+               dict(tile=4), dict(rounding=2), dict(alloc_tile=96), dict(hidden=32768, tile=128, alloc_tile=16384)]:
         p = T.Params(**{**base, **kw})
         assert T.packed_bound(p) == 0 and T.workspace_bound(p) == 0
         with pytest.raises(T.TahqError):
