@@ -1109,7 +1109,7 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const Args a) {
   }
   const int lane = threadIdx.x & 31;
 
-  // CTA 0 compares the received header with the one these parameters produce; its verdict travels
+  // CTA 0 compares the received header with the one these parameters produce; what it finds travels
   // with the offset prefix, so a refused buffer leaves the output untouched.
   bool refuse = false;
   if (blockIdx.x == 0) {

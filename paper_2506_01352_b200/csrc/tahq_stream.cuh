@@ -947,7 +947,7 @@ __global__ void __launch_bounds__(kThreads, 2) decode_stream_kernel(const Args a
   const uint64_t tile_cta = u0 * 32;
   const bool narrow = a.lo + a.mixed <= 4u;
 
-  // CTA 0 compares the received header with the one these parameters produce; its verdict travels
+  // CTA 0 compares the received header with the one these parameters produce; what it finds travels
   // with the offset prefix, so a refused buffer leaves the output untouched.
   bool refuse = false;
   if (blockIdx.x == 0) {
@@ -1066,7 +1066,7 @@ __global__ void __launch_bounds__(kThreads, 2) decode_stream_kernel(const Args a
     for (uint32_t i = threadIdx.x; i < nw; i += kThreads) s_bm[i] = bm_word(s0 + i);
     __syncthreads();
     const uint32_t seg_total = scan_segment(s_bm, nw, seg_hi, s_pre, s_wsum);
-    if (s0 == u0) {   // Sec. 3.4: higher-width tiles of all CTAs before this one; the header's verdict
+    if (s0 == u0) {   // Sec. 3.4: higher-width tiles of all CTAs before this one; what CTA 0 found in the header
       bool stop;
       const uint64_t mine = single ? (uint64_t)seg_total : counted;
       base_hi = cta_exclusive_prefix(a, mine, refuse, stop);
