@@ -845,11 +845,14 @@ __device__ __forceinline__ void dequant_narrow(const uint32_t (&wv)[N / 8], uint
   for (int j = 0; j < NG; ++j) {
     const uint32_t lo = g[j], hi = g[j] >> half;
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      uint32_t m;
-      asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(m) : "r"(i < 4 ? lo : hi), "r"(mk[i & 3]), "r"(two23));
-      const float f = __uint_as_float(m) - 8388608.0f;   // q * 2^p, exact
-      x[8 * j + i] = __fmaf_rn(f, sc[i & 3], z);
+    for (int i = 0; i < 8; i += 2) {   // two codes per packed instruction (same bits as the scalar operations)
+      uint32_t m0, m1;
+      asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(m0) : "r"(i < 4 ? lo : hi), "r"(mk[i & 3]), "r"(two23));
+      asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(m1) : "r"(i < 4 ? lo : hi), "r"(mk[(i + 1) & 3]), "r"(two23));
+      const float2 f = add2(f2(__uint_as_float(m0), __uint_as_float(m1)), f2(-8388608.0f));   // q * 2^p, exact
+      const float2 r = fma2(f, f2(sc[i & 3], sc[(i + 1) & 3]), f2(z));
+      x[8 * j + i] = r.x;
+      x[8 * j + i + 1] = r.y;
     }
   }
 }
