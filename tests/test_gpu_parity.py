@@ -118,6 +118,41 @@ def test_ragged_and_degenerate_shapes(shape, S, G, dtype):
         check_decode(p, packed, want, ws)
 
 
+def _random_case(k: int):
+    """Case k of a fixed pseudo-random sweep over the parameter space: shape, tile, group, budget, tau, dtype,
+    rounding mode and allocation tile all vary together."""
+    import random
+    r = random.Random(7919 * k + 13)
+    G = r.choice([8, 16, 32, 64, 128])
+    large = k >= 48                                        # ranking groups beyond the in-CTA selection, many CTAs
+    M = r.randint(16, 64) if large else r.randint(1, 24)   # tiles per token
+    m = r.choice([1, 1, 1] + [d for d in (2, 3, 4, 6, 8) if M % d == 0])
+    S = r.choice([250, 512, 777, 1000]) if large else r.choice([1, 2, 3, 5, 8, 16, 40, 96])
+    n_groups = r.randint(1, 4) if large else r.randint(1, 9)
+    tokens = S * n_groups
+    dtype = r.choice([torch.float32, torch.bfloat16])
+    beta = r.choice([2000, 2300, 2999, 3000, 3500, 3800, 4000, 4001, 5250, 6000, 7999, 8000])
+    tau = r.choice([0.0, 1.25, 2.0, 2.0, 2.0, 4.0, float("inf")])
+    rounding = r.choice([0, 0, 0, 1])
+    return dict(G=G, hidden=M * G, A=m * G, S=S, tokens=tokens, dtype=dtype, beta=beta, tau=tau, rounding=rounding,
+                seed=r.getrandbits(48), outliers=r.choice([0, 1, 3]), scale=r.choice([1e-3, 1.0, 40.0]))
+
+
+@pytest.mark.parametrize("k", range(64))
+def test_random_parameter_sweep(k):
+    c = _random_case(k)
+    g = torch.Generator(device="cuda").manual_seed(1000 + k)
+    x = torch.randn(c["tokens"], c["hidden"], generator=g, device="cuda")
+    x = x * torch.randn(c["tokens"], 1, generator=g, device="cuda").exp() * c["scale"]
+    for j in range(c["outliers"]):
+        x[:, (j * 29 + k) % c["hidden"]] *= 30
+    x = x.to(c["dtype"])
+    p = T.params_for(x, group_tokens=c["S"], tile=c["G"], budget_millibits=c["beta"], tau=c["tau"],
+                     rounding=c["rounding"], seed=c["seed"], alloc_tile=c["A"])
+    packed, want, ws = check_encode(p, x)
+    check_decode(p, packed, want, ws)
+
+
 @pytest.mark.parametrize("kind", ["zeros", "constant", "one_hot", "ties", "tau0", "tauinf", "huge"])
 def test_degenerate_values(kind):
     T_, C_ = 256, 512
