@@ -489,7 +489,9 @@ tahq_status tahq_decode(const tahq_params *p, const void *d_packed, size_t packe
   fill_args(p, pl, static_cast<uint8_t *>(d_ws), &a);
   a.packed = const_cast<uint8_t *>(static_cast<const uint8_t *>(d_packed));
   a.out = static_cast<uint8_t *>(d_out);
-  if (clear_workspace(d_ws, pl.ws_ncand, st) != TAHQ_OK) return TAHQ_ERR_CUDA;   // status + flags
+  // Up to 65536 bit-map words (256 KiB) the streaming kernel needs no look-back and nothing cleared: one launch.
+  a.own_prefix = p->tile != 128 && (pl.L.n_tiles + 31) / 32 <= 65536;
+  if (!a.own_prefix && clear_workspace(d_ws, pl.ws_ncand, st) != TAHQ_OK) return TAHQ_ERR_CUDA;   // status + flags
   const bool bf = p->dtype == TAHQ_BF16;
   switch (p->tile) {
     case 8: return bf ? decode_t<Cfg<8, true>>(pl, a, st) : decode_t<Cfg<8, false>>(pl, a, st);

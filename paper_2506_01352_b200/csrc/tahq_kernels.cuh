@@ -42,6 +42,7 @@ struct Args {
   uint32_t exact_scores;    // stats_kernel writes exact scores (small groups, or a varsigma too large to screen)
   unsigned long long *flags;// [kMaxGrid] (zeroed per call) per-CTA published counts for the offset prefix
   uint32_t use_tma;         // rows are 128 bytes and the tensor map is valid: units arrive by tiled TMA copies
+  uint32_t own_prefix;      // decode of a small tensor: every CTA counts the bit map before its slice itself
   uint32_t *gbar;           // [2] (zeroed per call) arrival counters of the fused encode kernel's grid barriers
   uint32_t *status;         // device status word
   unsigned long long seed;  // stochastic rounding mode: the generator's key

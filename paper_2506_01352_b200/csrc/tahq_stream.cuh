@@ -952,14 +952,16 @@ __global__ void __launch_bounds__(kThreads, 2) decode_stream_kernel(const Args a
 
   // CTA 0 compares the received header with the one these parameters produce; what it finds travels
   // with the offset prefix, so a refused buffer leaves the output untouched.
+  // (On a small tensor, a.own_prefix, every CTA does this itself and counts the bit map in front of its slice
+  // itself: no look-back, nothing that has to be cleared beforehand, one launch; the last CTA writes the status.)
   bool refuse = false;
-  if (blockIdx.x == 0) {
+  if (blockIdx.x == 0 || a.own_prefix) {
     if (threadIdx.x == 0) s_bad = 0;
     __syncthreads();
     if (threadIdx.x < 32 && reinterpret_cast<const uint32_t *>(a.packed)[threadIdx.x] != a.header[threadIdx.x]) s_bad = 1;
     __syncthreads();
     refuse = s_bad != 0;
-    if (refuse && threadIdx.x == 0) atomicOr(a.status, 1u /* TAHQ_DEV_BAD_HEADER */);
+    if (refuse && threadIdx.x == 0 && !a.own_prefix) atomicOr(a.status, 1u /* TAHQ_DEV_BAD_HEADER */);
   }
   // bit-map word i of the tensor, bits beyond the last tile cleared
   auto bm_word = [&](uint64_t i) -> uint32_t {
@@ -967,10 +969,20 @@ __global__ void __launch_bounds__(kThreads, 2) decode_stream_kernel(const Args a
     const uint64_t left = a.n_tiles - i * 32;
     return __ldg(bitmap + i) & (left >= 32 ? 0xffffffffu : ((1u << (uint32_t)left) - 1u));
   };
-  if (u0 == u1) {
+  if (u0 == u1) {   // (never the last CTA)
     bool stop;
-    cta_exclusive_prefix(a, 0, refuse, stop);
+    if (!a.own_prefix) cta_exclusive_prefix(a, 0, refuse, stop);
     return;
+  }
+  uint32_t own_before = 0;   // a.own_prefix: this thread's share of the higher-width tiles before the CTA's slice
+  if (a.own_prefix && a.mixed) {   // words before u0 are whole: 128-bit loads, then the last few one by one
+    const uint4 *b4 = reinterpret_cast<const uint4 *>(bitmap);
+    const uint64_t n4 = u0 / 4;
+    for (uint64_t i = threadIdx.x; i < n4; i += kThreads) {
+      const uint4 v = __ldg(b4 + i);
+      own_before += __popc(v.x) + __popc(v.y) + __popc(v.z) + __popc(v.w);
+    }
+    if (threadIdx.x < (uint32_t)(u0 - n4 * 4)) own_before += __popc(__ldg(bitmap + n4 * 4 + threadIdx.x));
   }
   const bool single = u1 - u0 <= (uint64_t)kSegWords;
   uint64_t counted = 0;
@@ -1072,9 +1084,17 @@ __global__ void __launch_bounds__(kThreads, 2) decode_stream_kernel(const Args a
     if (s0 == u0) {   // Sec. 3.4: higher-width tiles of all CTAs before this one; what CTA 0 found in the header
       bool stop;
       const uint64_t mine = single ? (uint64_t)seg_total : counted;
-      base_hi = cta_exclusive_prefix(a, mine, refuse, stop);
-      if (blockIdx.x == gridDim.x - 1 && threadIdx.x == 0 && a.mixed && !stop && base_hi + mine != a.n_groups * a.k_hi)
-        atomicOr(a.status, 2u /* TAHQ_DEV_BAD_BITMAP */);
+      if (a.own_prefix) {
+        base_hi = block_sum(refuse ? 0u : own_before);
+        stop = refuse;
+        if (blockIdx.x == gridDim.x - 1 && threadIdx.x == 0)
+          *a.status = (refuse ? 1u /* TAHQ_DEV_BAD_HEADER */ : 0u) |
+                      ((a.mixed && !refuse && base_hi + mine != a.n_groups * a.k_hi) ? 2u /* TAHQ_DEV_BAD_BITMAP */ : 0u);
+      } else {
+        base_hi = cta_exclusive_prefix(a, mine, refuse, stop);
+        if (blockIdx.x == gridDim.x - 1 && threadIdx.x == 0 && a.mixed && !stop && base_hi + mine != a.n_groups * a.k_hi)
+          atomicOr(a.status, 2u /* TAHQ_DEV_BAD_BITMAP */);
+      }
       if (stop) return;
       pay_off0 = (uint64_t)(C::G / 8) * ((uint64_t)a.lo * tile_cta + base_hi);
     }
