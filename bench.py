@@ -31,9 +31,9 @@ L2_BYTES = 126e6
 # profiles/ (same kernel, same workload); None until a capture exists for that kernel.
 NCU_TRAFFIC_BYTES = {
     # profiles/ncu_full_c3_llama7b_b3800_tile_kernels.md (cold-cache capture, one launch)
-    ("stats", "c3_llama7b", 3800, 64): 67.79e6,
-    ("quant_pack", "c3_llama7b", 3800, 64): 74.93e6,
-    ("decode", "c3_llama7b", 3800, 64): 27.91e6,
+    ("stats", "c3_llama7b", 3800, 64): 67.73e6,
+    ("quant_pack", "c3_llama7b", 3800, 64): 74.92e6,
+    ("decode", "c3_llama7b", 3800, 64): 27.94e6,
 }
 
 
