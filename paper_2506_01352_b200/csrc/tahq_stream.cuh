@@ -423,6 +423,19 @@ __device__ __forceinline__ void quant_phase(const Args &a, const void *tmap, uin
     }
   };
 
+  // The scores that the first rounds of the bit-map pass need are asked for first, into the slot that holds
+  // re-fetched rows later: left to that pass they are one load per thread and round, each waiting for the one
+  // before (0.45 us per round; the scores were written on the far side of the L2).
+  constexpr uint32_t kStagedRounds = S::UNIT_BYTES / 128;   // 32 scores per warp and round
+  const bool staged = !COH && a.mixed && a.alloc_m == 1;
+  float *const sc_stage = reinterpret_cast<float *>(fstage);
+  if (staged) {
+    const uint64_t t1 = (u0 + kSegWords < u1 ? u0 + kSegWords : u1) * 32;
+    uint32_t r = 0;
+    for (uint64_t t = u0 * 32 + threadIdx.x; t < t1 && t < a.n_tiles && r < kStagedRounds; t += kThreads, ++r)
+      cp_async4(sc_stage + r * 32 + lane, a.scores + t);
+    cp_async_commit();
+  }
   prime(u0, u0 + kSegWords < u1 ? u0 + kSegWords : u1);
 
   if (blockIdx.x == 0) {   // header and the zero padding behind every section
@@ -505,9 +518,17 @@ __device__ __forceinline__ void quant_phase(const Args &a, const void *tmap, uin
     if (a.mixed) {
       GroupCursor pc;
       pc.init(a, s0 * 32);
-      for (uint64_t tb = s0 * 32; tb < s1 * 32; tb += kThreads) {
+      const bool use_stage = staged && s0 == u0;
+      if (use_stage) {   // the scores asked for at the start (older than every group of the ring)
+        if (ring.tmap) cp_async_wait<0>();
+        else cp_async_wait<NST>();
+      }
+      uint32_t r = 0;
+      for (uint64_t tb = s0 * 32; tb < s1 * 32; tb += kThreads, ++r) {
         const uint64_t t = tb + threadIdx.x;
-        const bool hi = t < a.n_tiles && pc.template is_hi<COH>(a, t, threadIdx.x);
+        const bool hi = t < a.n_tiles && ((use_stage && r < kStagedRounds)
+                                              ? pc.is_hi_score(a, sc_stage[r * 32 + lane], threadIdx.x)
+                                              : pc.template is_hi<COH>(a, t, threadIdx.x));
         const unsigned word = __ballot_sync(kFull, hi);
         if (lane == 0 && (t >> 5) < s1) {
           s_bm[(t >> 5) - s0] = word;
