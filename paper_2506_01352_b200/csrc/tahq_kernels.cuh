@@ -112,8 +112,9 @@ __device__ __forceinline__ uint64_t cta_exclusive_prefix(const Args &a, uint64_t
   __shared__ uint32_t s_abort;
   if (threadIdx.x == 0) {
     s_abort = 0;
-    __threadfence();
-    atomicExch(a.flags + blockIdx.x, kPublished | (abort_in ? kAbort : 0ull) | (mine & kCountMask));
+    // one aligned 64-bit store: the word carries everything that is published, so nothing has to be fenced
+    *reinterpret_cast<volatile unsigned long long *>(a.flags + blockIdx.x) =
+        kPublished | (abort_in ? kAbort : 0ull) | (mine & kCountMask);
   }
   __syncthreads();
   unsigned long long sum = 0;
