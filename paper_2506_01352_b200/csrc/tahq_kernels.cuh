@@ -527,21 +527,89 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const Args a) {
   (void)r;
   const unsigned long long *cand = a.cand + g * a.cand_cap;
   unsigned long long t;
-  if (n <= a.cand_cap && n <= (uint32_t)kSelThreads) {
-    // few candidates (the usual case): every thread ranks one key by counting the larger ones
-    const unsigned long long mine = threadIdx.x < n ? __ldcg(cand + threadIdx.x) : 0ull;
-    s_keys[threadIdx.x] = mine;
+  if (n <= a.cand_cap) {
+    // The candidates are all in the list (the usual case); up to kSortCap - kSelThreads of them are copied to
+    // shared memory.  A handful are ranked by counting, for every key, the larger ones.  More (a threshold in the
+    // dense part of the scores: hundreds to thousands per group) first go into kSelThreads buckets by score,
+    // spread evenly between the smallest and the largest; the bucket that holds rank rr is found by a suffix sum
+    // and only its few keys are counted against each other.
+    const bool in_smem = n <= (uint32_t)(kSortCap - kSelThreads);
+    if (in_smem) {
+      for (uint32_t i = threadIdx.x; i < n; i += kSelThreads) s_keys[i] = __ldcg(cand + i);
+      __syncthreads();
+    }
+    if (n <= 64u) {
+      if (threadIdx.x >= n) return;
+      const unsigned long long mine = s_keys[threadIdx.x];
+      uint32_t larger = 0;
+      for (uint32_t i = 0; i < n; ++i) larger += s_keys[i] > mine ? 1u : 0u;
+      if (larger == rr - 1) a.theta[g] = mine;   // keys are distinct: exactly one thread
+      return;
+    }
+    auto key_at = [&](uint32_t i) { return in_smem ? s_keys[i] : __ldcg(cand + i); };
+    __shared__ uint32_t s_cnt[kSelThreads];   // keys per bucket
+    __shared__ uint32_t s_sub[kSelThreads];   // the keys (their indices) of the bucket that holds rank rr
+    __shared__ uint32_t s_lo, s_hi, s_nsub;
+    if (threadIdx.x == 0) { s_lo = 0xffffffffu; s_hi = 0; s_nsub = 0; s_sel[0] = 0; s_sel[1] = 0; }
+    s_cnt[threadIdx.x] = 0;
     __syncthreads();
-    uint32_t larger = 0;
-    for (uint32_t i = 0; i < n; ++i) larger += s_keys[i] > mine ? 1u : 0u;
-    if (threadIdx.x < n && larger == rr - 1) a.theta[g] = mine;   // keys are distinct: exactly one thread
-    return;
-  } else if (n <= a.cand_cap && n <= (uint32_t)kSortCap) {
-    for (uint32_t i = threadIdx.x; i < n; i += kSelThreads) s_keys[i] = __ldcg(cand + i);
+    {   // the scores, mapped to unsigned integers of the same order: smallest and largest
+      uint32_t mn = 0xffffffffu, mx = 0;
+      for (uint32_t i = threadIdx.x; i < n; i += kSelThreads) {
+        const uint32_t m = (uint32_t)(key_at(i) >> 32);
+        mn = m < mn ? m : mn;
+        mx = m > mx ? m : mx;
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        const uint32_t v = __shfl_xor_sync(kFull, mn, o), w = __shfl_xor_sync(kFull, mx, o);
+        mn = v < mn ? v : mn;
+        mx = w > mx ? w : mx;
+      }
+      if (lane == 0) { atomicMin(&s_lo, mn); atomicMax(&s_hi, mx); }
+    }
     __syncthreads();
-    t = radix_select(n, rr, from_smem);
-  } else if (n <= a.cand_cap) {
-    t = radix_select(n, rr, [&](uint64_t i, unsigned long long &key) {
+    const uint32_t lo_m = s_lo, span = s_hi - s_lo;
+    auto bucket_of = [&](unsigned long long key) {
+      return span ? (uint32_t)(((unsigned long long)((uint32_t)(key >> 32) - lo_m) * (kSelThreads - 1)) / span) : 0u;
+    };
+    for (uint32_t i = threadIdx.x; i < n; i += kSelThreads) atomicAdd(&s_cnt[bucket_of(key_at(i))], 1u);
+    __syncthreads();
+    {   // keys in the buckets above this thread's bucket (one bucket per thread)
+      const uint32_t c = s_cnt[threadIdx.x];
+      uint32_t incl = c;
+#pragma unroll
+      for (int o = 1; o < 32; o *= 2) {
+        const uint32_t v = __shfl_down_sync(kFull, incl, o);
+        if (lane + o < 32) incl += v;
+      }
+      if (lane == 0) s_warp[warp] = incl;
+      __syncthreads();
+      uint32_t above = incl - c;
+      for (int w = warp + 1; w < kSelThreads / 32; ++w) above += s_warp[w];
+      if (above < rr && above + c >= rr) { s_sel[0] = threadIdx.x; s_sel[1] = rr - above; }
+    }
+    __syncthreads();
+    const uint32_t bsel = s_sel[0], rsel = s_sel[1];
+    if (rsel != 0 && s_cnt[bsel] <= (uint32_t)kSelThreads) {
+      for (uint32_t i = threadIdx.x; i < n; i += kSelThreads)
+        if (bucket_of(key_at(i)) == bsel) s_sub[atomicAdd(&s_nsub, 1u)] = i;
+      __syncthreads();
+      const uint32_t ns = s_nsub;
+      unsigned long long *s_few = s_keys + kSortCap - kSelThreads;   // the bucket's keys, behind the copied ones
+      const unsigned long long mine = threadIdx.x < ns ? key_at(s_sub[threadIdx.x]) : 0ull;
+      if (threadIdx.x < ns) s_few[threadIdx.x] = mine;
+      __syncthreads();
+      if (threadIdx.x < ns) {
+        uint32_t larger = 0;
+        for (uint32_t i = 0; i < ns; ++i) larger += s_few[i] > mine ? 1u : 0u;
+        if (larger == rsel - 1) a.theta[g] = mine;   // keys are distinct: exactly one thread
+      }
+      return;
+    }
+    // thousands of equal scores: bit by bit
+    if (in_smem) t = radix_select(n, rr, from_smem);
+    else t = radix_select(n, rr, [&](uint64_t i, unsigned long long &key) {
       key = __ldcg(cand + i);
       return true;
     });
