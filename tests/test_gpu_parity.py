@@ -208,6 +208,31 @@ def test_selection_with_near_tied_scores(eps_log):
     check_decode(p, packed, want, ws)
 
 
+@pytest.mark.parametrize("kind", ["thousands", "ten_thousand", "equal_by_the_thousand", "more_than_the_list_holds"])
+def test_selection_with_many_candidates(kind):
+    """A threshold in the middle of a narrow score distribution: thousands of candidates next to it (ranked in
+    shared memory), about ten thousand (ranked from the list in global memory), thousands of exactly equal scores
+    among them (buckets cannot separate those), and more candidates than the list holds (the group's stored scores
+    are ranked instead)."""
+    g = torch.Generator(device="cuda").manual_seed(4242 + len(kind))
+    if kind == "more_than_the_list_holds":
+        base = torch.randn(64, generator=g, device="cuda")
+        perm = torch.rand(40000, 64, generator=g, device="cuda").argsort(1)
+        x = base[perm] * (1.0 + 1e-4 * torch.randn(40000, 64, generator=g, device="cuda"))
+        x = x.reshape(1250, 2048)
+    else:
+        tokens = 8192 if kind == "ten_thousand" else 2048
+        x = torch.randn(tokens, 4096, generator=g, device="cuda")
+        if kind == "equal_by_the_thousand":
+            tiles = x.view(-1, 64)
+            mid = tiles[torch.argsort(tiles.abs().sum(1))[tiles.shape[0] // 2]].clone()
+            tiles[5:5 + 3 * 6000:3] = mid
+        x = x.to(torch.bfloat16)
+    p = T.params_for(x, group_tokens=0, tile=64, budget_millibits=3500)
+    packed, want, ws = check_encode(p, x)
+    check_decode(p, packed, want, ws)
+
+
 @pytest.mark.parametrize("G", [8, 16, 32, 64, 128])
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
 def test_stochastic_rounding_mode(G, dtype):
