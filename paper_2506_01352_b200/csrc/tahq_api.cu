@@ -241,7 +241,13 @@ static cudaError_t launch_dependent(void (*kernel)(P...), unsigned grid, unsigne
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, kernel, std::forward<A>(args)...);
+  cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, args...);
+  if (e == cudaErrorNotSupported || e == cudaErrorInvalidValue) {   // attribute refused: an ordinary launch does
+    (void)cudaGetLastError();
+    cfg.numAttrs = 0;
+    e = cudaLaunchKernelEx(&cfg, kernel, args...);
+  }
+  return e;
 }
 
 // Zero the first `bytes` (a multiple of 16) of the workspace with a kernel, so that the call's next kernel can
