@@ -371,11 +371,19 @@ static tahq_status encode_t(const Plan &pl, const Args &a_in, cudaStream_t st) {
   if constexpr (C::LPT == 1) {   // one lane per tile: warps stream units of 32 tiles independently
     constexpr int NQ = 2;
     const int smem = StreamCfg<C>::smem_bytes(NQ);
-    const int occ = prepare(quant_pack_stream_kernel<C, NQ, SR>, smem, d, occ_quant);
+    static std::atomic<int> occ_wide[64];
+    const bool narrow = a.lo + a.mixed <= 4u;   // no width above 4 bits: the kernel compiled for just that
+    const int occ = narrow ? prepare(quant_pack_stream_kernel<C, NQ, SR, true>, smem, d, occ_quant)
+                           : prepare(quant_pack_stream_kernel<C, NQ, SR, false>, smem, d, occ_wide);
     if (!occ) return TAHQ_ERR_CUDA;
     const uint64_t n_units = (a.n_tiles + 31) / 32;
     const unsigned grid = persistent_grid((n_units + kWarps - 1) / kWarps, d, occ);
-    TAHQ_LAUNCH("quant_pack", st, launch_dependent(quant_pack_stream_kernel<C, NQ, SR>, grid, kThreads, smem, st, a, tmap));
+    if (narrow)
+      TAHQ_LAUNCH("quant_pack", st,
+                  launch_dependent(quant_pack_stream_kernel<C, NQ, SR, true>, grid, kThreads, smem, st, a, tmap));
+    else
+      TAHQ_LAUNCH("quant_pack", st,
+                  launch_dependent(quant_pack_stream_kernel<C, NQ, SR, false>, grid, kThreads, smem, st, a, tmap));
   } else {
     constexpr int NQ = Stages<C>::QUANT;
     const int smem = NQ * (C::STAGE_BYTES + C::TPC * 4);
