@@ -345,12 +345,16 @@ static tahq_status encode_t(const Plan &pl, const Args &a_in, cudaStream_t st) {
     } else if constexpr (C::LPT == 1) {
       constexpr int NS = C::ROWB <= 128 ? 3 : 2;
       const int smem = kWarps * NS * StreamCfg<C>::UNIT_BYTES + 256;   // ring slots, then the warps' mbarriers
-      const int occ = prepare(stats_stream_kernel<C, NS>, smem, d, occ_stats);
+      static std::atomic<int> occ_exact[64];
+      const int occ = a.exact_scores ? prepare(stats_stream_kernel<C, NS, true>, smem, d, occ_exact)
+                                     : prepare(stats_stream_kernel<C, NS, false>, smem, d, occ_stats);
       if (!occ) return TAHQ_ERR_CUDA;
       const uint64_t n_units = (a.n_tiles + 31) / 32;
-      TAHQ_LAUNCH("stats", st,
-                  launch_dependent(stats_stream_kernel<C, NS>, persistent_grid((n_units + kWarps - 1) / kWarps, d, occ),
-                                   kThreads, smem, st, a, tmap));
+      const unsigned grid = persistent_grid((n_units + kWarps - 1) / kWarps, d, occ);
+      if (a.exact_scores)
+        TAHQ_LAUNCH("stats", st, launch_dependent(stats_stream_kernel<C, NS, true>, grid, kThreads, smem, st, a, tmap));
+      else
+        TAHQ_LAUNCH("stats", st, launch_dependent(stats_stream_kernel<C, NS, false>, grid, kThreads, smem, st, a, tmap));
     } else {
       constexpr int NS = Stages<C>::STATS;
       const int smem = NS * C::STAGE_BYTES;

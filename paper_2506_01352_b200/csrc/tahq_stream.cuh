@@ -161,7 +161,8 @@ __device__ __forceinline__ void words_minmax(const uint32_t (&w)[C::ROWB / 4], f
 // ------------------------------------------------------------------------------------------
 // Eq. 1-2, warp-streaming: entropy score per tile, per-group histogram of binned scores (Sec. 3.2)
 // ------------------------------------------------------------------------------------------
-template <class C, int NST>
+// SCORE: 0 = screening scores, 1 = exact scores, 2 = whichever the call asks for (a.exact_scores)
+template <class C, int NST, int SCORE>
 __device__ __forceinline__ void stats_phase(const Args &a, const void *tmap, uint8_t *smem, unsigned long long *bars,
                                             uint32_t *s_hist) {
   using S = StreamCfg<C>;
@@ -198,8 +199,9 @@ __device__ __forceinline__ void stats_phase(const Args &a, const void *tmap, uin
       ring.wait(a, slot);
       const uint8_t *stage = ring.slot(slot);
       // small groups are ranked on exact scores; large ones are screened first (see select_kernel)
-      const float s = a.exact_scores ? tile_score<C>(stage, lane, a.eps_l1, a.eps_log)
-                                     : tile_score_screen<C>(stage, lane, a.eps_l1);
+      const bool exact = SCORE == 2 ? a.exact_scores != 0 : SCORE == 1;
+      const float s = exact ? tile_score<C>(stage, lane, a.eps_l1, a.eps_log)
+                            : tile_score_screen<C>(stage, lane, a.eps_l1);
       __syncwarp();
       {
         const uint64_t kn = k + (uint64_t)NST * kWarps;
@@ -229,13 +231,13 @@ __device__ __forceinline__ void stats_phase(const Args &a, const void *tmap, uin
   }
 }
 
-template <class C, int NST>
+template <class C, int NST, bool EXACT>
 __global__ void __launch_bounds__(kThreads, 2) stats_stream_kernel(const Args a, const __grid_constant__ CUtensorMap tmap) {
   extern __shared__ __align__(1024) uint8_t smem_1k[];
   uint8_t *smem = smem_1k;
   __shared__ uint32_t s_hist[kBins];   // this CTA's counts for the ranking group it is in
   grid_dependency_wait();   // the histograms are cleared by the kernel in front
-  stats_phase<C, NST>(a, &tmap, smem, reinterpret_cast<unsigned long long *>(smem + (size_t)kWarps * NST * StreamCfg<C>::UNIT_BYTES),
+  stats_phase<C, NST, EXACT ? 1 : 0>(a, &tmap, smem, reinterpret_cast<unsigned long long *>(smem + (size_t)kWarps * NST * StreamCfg<C>::UNIT_BYTES),
                       s_hist);
 }
 
@@ -801,7 +803,7 @@ __global__ void __launch_bounds__(kThreads, 2) encode_fused_kernel(const Args a,
   extern __shared__ __align__(1024) uint8_t smem_1k[];
   uint8_t *smem = smem_1k;
   // Eq. 1-2: two ring slots per warp, the CTA's histogram behind them; mbarriers at the very end
-  stats_phase<C, 2>(a, &tmap, smem,
+  stats_phase<C, 2, 2>(a, &tmap, smem,
                     reinterpret_cast<unsigned long long *>(smem + (size_t)kWarps * 3 * S::UNIT_BYTES + 128),
                     reinterpret_cast<uint32_t *>(smem + (size_t)kWarps * 2 * S::UNIT_BYTES));
   grid_barrier(a, 0);   // every histogram is complete
