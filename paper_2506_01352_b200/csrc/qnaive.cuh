@@ -71,6 +71,172 @@ __global__ void __launch_bounds__(kQThreads) qnaive_max_kernel(const QArgs a) {
   if ((threadIdx.x & 31) == 0 && m > 0.0f) atomicMax(a.gmax, __float_as_uint(m));
 }
 
+// ---- rows of whole kilo-elements at 6 or 8 bits (the widths the paper runs the backward half at) -------------
+// A lane owns 32 consecutive elements of every 1024: they arrive by 128-bit loads and stay in registers as
+// loaded; four codes are glued by a multiply-add chain on the raw bits of fma(y, 1/s, 1.5 * 2^23) (the
+// constant part of those bits, less L per code, is taken off once per chain), and the lane's 24 or 32 bytes
+// leave by 64- or 128-bit stores.  The clamp of the general path is left out: |y| <= m and s = m / L rounded
+// give |y * (1/s)| < L + 1/2, so it never acts on finite input.  Same bytes as the general path.
+template <bool BF16>
+struct QFast {
+  static constexpr int V = BF16 ? 4 : 8;        // 128-bit pieces holding a lane's 32 elements of one kilo-element
+  static constexpr int NCH = BF16 ? 4 : 2;      // kilo-elements a row may have (64 registers of raw data)
+  __device__ static __forceinline__ float elem(const uint4 (&raw)[V], int e) {
+    if constexpr (BF16) {
+      const uint4 &q = raw[e / 8];
+      const int wsel = (e % 8) / 2;
+      const uint32_t w = wsel == 0 ? q.x : wsel == 1 ? q.y : wsel == 2 ? q.z : q.w;
+      return (e & 1) ? __uint_as_float(w & 0xffff0000u) : __uint_as_float(w << 16);
+    } else {
+      const uint4 &q = raw[e / 4];
+      const int wsel = e % 4;
+      return __uint_as_float(wsel == 0 ? q.x : wsel == 1 ? q.y : wsel == 2 ? q.z : q.w);
+    }
+  }
+};
+
+template <bool BF16, int B>
+__device__ __forceinline__ void qnaive_encode_rows_fast(const QArgs &a, int lane, uint64_t warp, uint64_t n_warps) {
+  using F = QFast<BF16>;
+  constexpr int ESZ = BF16 ? 2 : 4;
+  constexpr int Lq = (1 << (B - 1)) - 1;
+  constexpr uint32_t kMb = 0x4B400000u;   // bits of 1.5 * 2^23
+  constexpr uint32_t kOnes = B == 6 ? (1u + (1u << 6) + (1u << 12) + (1u << 18)) : (1u + (1u << 8) + (1u << 16) + (1u << 24));
+  constexpr uint32_t kOff = (uint32_t)(((unsigned long long)(kMb - (uint32_t)Lq) * kOnes) & 0xffffffffull);
+  uint32_t M = 1u << B;
+  asm volatile("mov.u32 %0, %0;" : "+r"(M));   // opaque: the chain stays one multiply-add per code
+  const uint32_t C = a.hidden, nch = C / 1024u;
+  float *scales = reinterpret_cast<float *>(a.packed + a.off_scales);
+  for (uint64_t r = warp; r < a.tokens; r += n_warps) {
+    const uint8_t *row = a.in + (r * (uint64_t)C + (uint64_t)lane * 32u) * ESZ;
+    uint8_t *orow = a.packed + a.off_payload + r * a.row_bytes;
+    uint4 raw[F::NCH][F::V];
+#pragma unroll
+    for (int ch = 0; ch < F::NCH; ++ch)
+#pragma unroll
+      for (int v = 0; v < F::V; ++v)
+        raw[ch][v] = (uint32_t)ch < nch ? __ldg(reinterpret_cast<const uint4 *>(row + (size_t)ch * 1024 * ESZ) + v)
+                                        : make_uint4(0, 0, 0, 0);
+    float m = 0.0f;
+    if (a.per_tensor) {
+      m = __uint_as_float(*a.gmax);
+    } else {
+#pragma unroll
+      for (int ch = 0; ch < F::NCH; ++ch)
+#pragma unroll
+        for (int e = 0; e < 32; ++e) m = fmaxf(m, fabsf(a.prescale * F::elem(raw[ch], e)));   // (zeros beyond the row)
+      m = warp_max(m);
+    }
+    const float s = __fdiv_rn(m, (float)Lq);
+    const float inv = s > 0.0f ? __frcp_rn(s) : 0.0f;
+    if (lane == 0 && (!a.per_tensor || r == 0)) scales[a.per_tensor ? 0 : r] = s;
+#pragma unroll
+    for (int ch = 0; ch < F::NCH; ++ch) {
+      if ((uint32_t)ch < nch) {
+        uint32_t g[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          uint32_t acc = 0;
+#pragma unroll
+          for (int k = 3; k >= 0; --k) {
+            const float y = a.prescale * F::elem(raw[ch], 4 * j + k);
+            const uint32_t bits = __float_as_uint(__fmaf_rn(y, inv, kQMagic));   // one rounding, ties to even
+            acc = k == 3 ? bits : acc * M + bits;
+          }
+          g[j] = acc - kOff;
+        }
+        if constexpr (B == 8) {
+          uint4 *dst = reinterpret_cast<uint4 *>(orow + (size_t)ch * 1024 + (size_t)lane * 32);
+          dst[0] = make_uint4(g[0], g[1], g[2], g[3]);
+          dst[1] = make_uint4(g[4], g[5], g[6], g[7]);
+        } else {
+          uint32_t w[6];
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            w[3 * h] = __byte_perm(g[4 * h], g[4 * h + 1], 0x4210);
+            w[3 * h + 1] = __byte_perm(g[4 * h + 1], g[4 * h + 2], 0x5421);
+            w[3 * h + 2] = __byte_perm(g[4 * h + 2], g[4 * h + 3], 0x6542);
+          }
+          uint2 *dst = reinterpret_cast<uint2 *>(orow + (size_t)ch * 768 + (size_t)lane * 24);
+#pragma unroll
+          for (int j = 0; j < 3; ++j) dst[j] = make_uint2(w[2 * j], w[2 * j + 1]);
+        }
+      }
+    }
+  }
+}
+
+template <bool BF16, int B>
+__device__ __forceinline__ void qnaive_decode_rows_fast(const QArgs &a, int lane, uint64_t warp, uint64_t n_warps,
+                                                        bool pow2, float rc) {
+  constexpr int ESZ = BF16 ? 2 : 4;
+  constexpr int Lq = (1 << (B - 1)) - 1;
+  constexpr uint32_t kMb = 0x4B400000u;
+  const float off = kQMagic + (float)Lq;   // exact
+  const uint32_t C = a.hidden, nch = C / 1024u;
+  const float *scales = reinterpret_cast<const float *>(a.packed + a.off_scales);
+  for (uint64_t r = warp; r < a.tokens; r += n_warps) {
+    const float s = __ldg(scales + (a.per_tensor ? 0 : r));
+    const uint8_t *irow = a.packed + a.off_payload + r * a.row_bytes;
+    uint8_t *orow = a.out + (r * (uint64_t)C + (uint64_t)lane * 32u) * ESZ;
+    for (uint32_t ch = 0; ch < nch; ++ch) {
+      uint32_t g[8];   // four codes each
+      if constexpr (B == 8) {
+        const uint4 *src = reinterpret_cast<const uint4 *>(irow + (size_t)ch * 1024 + (size_t)lane * 32);
+        const uint4 v0 = __ldg(src), v1 = __ldg(src + 1);
+        g[0] = v0.x; g[1] = v0.y; g[2] = v0.z; g[3] = v0.w;
+        g[4] = v1.x; g[5] = v1.y; g[6] = v1.z; g[7] = v1.w;
+      } else {
+        const uint2 *src = reinterpret_cast<const uint2 *>(irow + (size_t)ch * 768 + (size_t)lane * 24);
+        uint32_t w[6];
+#pragma unroll
+        for (int j = 0; j < 3; ++j) {
+          const uint2 v = __ldg(src + j);
+          w[2 * j] = v.x;
+          w[2 * j + 1] = v.y;
+        }
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {   // 24 bits per group, in its low three bytes
+          g[4 * h] = w[3 * h];
+          g[4 * h + 1] = __byte_perm(w[3 * h], w[3 * h + 1], 0x5543);
+          g[4 * h + 2] = __byte_perm(w[3 * h + 1], w[3 * h + 2], 0x4432);
+          g[4 * h + 3] = w[3 * h + 2] >> 8;
+        }
+      }
+      float x[32];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          uint32_t mbits;   // the code in the mantissa of 1.5 * 2^23
+          if constexpr (B == 8) mbits = __byte_perm(g[j], kMb, 0x7640 + k);
+          else mbits = ((g[j] >> (6 * k)) & 63u) | kMb;
+          const float q = __uint_as_float(mbits) - off;   // code - L, exact
+          const float t = __fmul_rn(q, s);
+          x[4 * j + k] = pow2 ? __fmul_rn(t, rc) : __fdiv_rn(t, a.prescale);
+        }
+      }
+      uint8_t *dst = orow + (size_t)ch * 1024 * ESZ;
+      if constexpr (BF16) {
+#pragma unroll
+        for (int v = 0; v < 4; ++v) {
+          uint32_t u[4];
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const __nv_bfloat162 h2 = __floats2bfloat162_rn(x[8 * v + 2 * j], x[8 * v + 2 * j + 1]);
+            u[j] = *reinterpret_cast<const uint32_t *>(&h2);
+          }
+          reinterpret_cast<uint4 *>(dst)[v] = make_uint4(u[0], u[1], u[2], u[3]);
+        }
+      } else {
+#pragma unroll
+        for (int v = 0; v < 8; ++v)
+          reinterpret_cast<float4 *>(dst)[v] = make_float4(x[4 * v], x[4 * v + 1], x[4 * v + 2], x[4 * v + 3]);
+      }
+    }
+  }
+}
+
 template <bool BF16>
 __global__ void __launch_bounds__(kQThreads, 2) qnaive_encode_kernel(const QArgs a) {
   grid_dependency_wait();   // launched as a programmatic dependent of the kernel in front
@@ -88,6 +254,11 @@ __global__ void __launch_bounds__(kQThreads, 2) qnaive_encode_kernel(const QArgs
     const uint64_t n_s = a.per_tensor ? 1 : a.tokens;
     for (uint64_t o = a.off_scales + 4 * n_s + threadIdx.x; o < a.off_payload; o += kQThreads) a.packed[o] = 0;
     for (uint64_t o = a.off_payload + a.tokens * a.row_bytes + threadIdx.x; o < a.total_bytes; o += kQThreads) a.packed[o] = 0;
+  }
+  if ((b == 6u || b == 8u) && C % 1024u == 0u && C <= (uint32_t)QFast<BF16>::NCH * 1024u) {
+    if (b == 6u) qnaive_encode_rows_fast<BF16, 6>(a, lane, warp, n_warps);
+    else qnaive_encode_rows_fast<BF16, 8>(a, lane, warp, n_warps);
+    return;
   }
   const uint32_t data_bytes = (uint32_t)(((uint64_t)C * b) >> 3);   // hidden is a multiple of 8
   // pieces a lane's b bytes are stored in: the largest power of two dividing b, at most 16
@@ -269,6 +440,11 @@ __global__ void __launch_bounds__(kQThreads) qnaive_decode_kernel(const QArgs a)
   // dividing by a power of two is the same rounding as multiplying by its (exact) reciprocal
   const bool pow2 = (__float_as_uint(a.prescale) & 0x007fffffu) == 0u && (__float_as_uint(a.prescale) >> 23) - 2u < 250u;
   const float rc = pow2 ? __frcp_rn(a.prescale) : 0.0f;
+  if ((b == 6u || b == 8u) && C % 1024u == 0u) {
+    if (b == 6u) qnaive_decode_rows_fast<BF16, 6>(a, lane, warp, n_warps, pow2, rc);
+    else qnaive_decode_rows_fast<BF16, 8>(a, lane, warp, n_warps, pow2, rc);
+    return;
+  }
   for (uint64_t r = warp; r < a.tokens; r += n_warps) {
     const float s = __ldg(scales + (a.per_tensor ? 0 : r));
     const uint8_t *irow = a.packed + a.off_payload + r * a.row_bytes;

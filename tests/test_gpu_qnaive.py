@@ -51,6 +51,20 @@ def test_ragged_shapes_and_dtypes(shape, dtype):
     _check(x, 6, 1, 1.0)
 
 
+@pytest.mark.parametrize("shape", [(5, 1024), (9, 2048), (4, 3072), (300, 4096), (3, 5120)])
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_rows_of_whole_kilo_elements(shape, dtype):
+    """6 and 8 bits on rows of n x 1024 elements take kernels of their own (a lane owns 32 consecutive elements);
+    (3, 5120) is past what they hold in registers when encoding."""
+    g = torch.Generator(device="cuda").manual_seed(shape[0] * 7 + shape[1])
+    x = torch.randn(shape, generator=g, device="cuda") * torch.randn(shape[0], 1, generator=g, device="cuda").exp() * 1e-3
+    x = x.to(dtype)
+    x[-1] = 0
+    for bits in (6, 8):
+        for per_tensor, c in ((0, 1024.0), (0, 3.0), (1, 1.0)):
+            _check(x, bits, per_tensor, c)
+
+
 def test_llama_shaped_gradient_bf16():
     x = (synth.make("c3_llama7b", device="cuda").float() * 1e-4).to(torch.bfloat16)
     _check(x, 6, 0, 4096.0)
