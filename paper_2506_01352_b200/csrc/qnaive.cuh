@@ -166,9 +166,9 @@ __device__ __forceinline__ void qnaive_encode_rows_fast(const QArgs &a, int lane
   }
 }
 
-template <bool BF16, int B>
+template <bool BF16, int B, bool POW2>
 __device__ __forceinline__ void qnaive_decode_rows_fast(const QArgs &a, int lane, uint64_t warp, uint64_t n_warps,
-                                                        bool pow2, float rc) {
+                                                        float rc) {
   constexpr int ESZ = BF16 ? 2 : 4;
   constexpr int Lq = (1 << (B - 1)) - 1;
   constexpr uint32_t kMb = 0x4B400000u;
@@ -178,7 +178,6 @@ __device__ __forceinline__ void qnaive_decode_rows_fast(const QArgs &a, int lane
   for (uint64_t r = warp; r < a.tokens; r += n_warps) {
     const float s = __ldg(scales + (a.per_tensor ? 0 : r));
     const uint8_t *irow = a.packed + a.off_payload + r * a.row_bytes;
-    uint8_t *orow = a.out + (r * (uint64_t)C + (uint64_t)lane * 32u) * ESZ;
     for (uint32_t ch = 0; ch < nch; ++ch) {
       uint32_t g[8];   // four codes each
       if constexpr (B == 8) {
@@ -213,25 +212,54 @@ __device__ __forceinline__ void qnaive_decode_rows_fast(const QArgs &a, int lane
           else mbits = ((g[j] >> (6 * k)) & 63u) | kMb;
           const float q = __uint_as_float(mbits) - off;   // code - L, exact
           const float t = __fmul_rn(q, s);
-          x[4 * j + k] = pow2 ? __fmul_rn(t, rc) : __fdiv_rn(t, a.prescale);
+          x[4 * j + k] = POW2 ? __fmul_rn(t, rc) : __fdiv_rn(t, a.prescale);
         }
       }
-      uint8_t *dst = orow + (size_t)ch * 1024 * ESZ;
+      // The lane's 32 values as 128-bit pieces.  Neighbouring lanes swap half of them (the even lane's odd pieces
+      // against the odd lane's even ones), so that the two lanes of a pair write 32 adjacent bytes in every store
+      // instruction: stored as they are, each instruction would write half of every 32-byte sector it touches.
+      constexpr int V = BF16 ? 4 : 8;
+      uint4 pc[V];
       if constexpr (BF16) {
 #pragma unroll
-        for (int v = 0; v < 4; ++v) {
+        for (int v = 0; v < V; ++v) {
           uint32_t u[4];
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
             const __nv_bfloat162 h2 = __floats2bfloat162_rn(x[8 * v + 2 * j], x[8 * v + 2 * j + 1]);
             u[j] = *reinterpret_cast<const uint32_t *>(&h2);
           }
-          reinterpret_cast<uint4 *>(dst)[v] = make_uint4(u[0], u[1], u[2], u[3]);
+          pc[v] = make_uint4(u[0], u[1], u[2], u[3]);
         }
       } else {
 #pragma unroll
-        for (int v = 0; v < 8; ++v)
-          reinterpret_cast<float4 *>(dst)[v] = make_float4(x[4 * v], x[4 * v + 1], x[4 * v + 2], x[4 * v + 3]);
+        for (int v = 0; v < V; ++v)
+          pc[v] = make_uint4(__float_as_uint(x[4 * v]), __float_as_uint(x[4 * v + 1]), __float_as_uint(x[4 * v + 2]),
+                             __float_as_uint(x[4 * v + 3]));
+      }
+      const bool odd = lane & 1;
+#pragma unroll
+      for (int h = 0; h < V / 2; ++h) {   // even lane: gives piece 2h+1, gets the neighbour's piece 2h; odd lane: the reverse
+        const uint4 give = odd ? pc[2 * h] : pc[2 * h + 1];
+        uint4 got;
+        got.x = __shfl_xor_sync(0xffffffffu, give.x, 1);
+        got.y = __shfl_xor_sync(0xffffffffu, give.y, 1);
+        got.z = __shfl_xor_sync(0xffffffffu, give.z, 1);
+        got.w = __shfl_xor_sync(0xffffffffu, give.w, 1);
+        if (odd) pc[2 * h] = got; else pc[2 * h + 1] = got;
+      }
+      // now: even lane holds its own even pieces and the neighbour's even pieces (at the odd slots); the odd lane
+      // its own odd pieces (odd slots) and the neighbour's odd pieces (even slots)
+      uint8_t *pair0 = a.out + (r * (uint64_t)C + (uint64_t)(lane & ~1) * 32u + (uint64_t)ch * 1024u) * ESZ;
+#pragma unroll
+      for (int h = 0; h < V / 2; ++h) {
+        // pieces 2h and 2h+1 of the even lane's region, then of the odd lane's region
+        uint4 *even_region = reinterpret_cast<uint4 *>(pair0) + 2 * h;
+        uint4 *odd_region = reinterpret_cast<uint4 *>(pair0 + 32 * ESZ) + 2 * h;
+        // even lane: its own piece 2h, then the neighbour's piece 2h; odd lane: the neighbour's piece 2h+1, then
+        // its own piece 2h+1 (one instruction for both lanes, so each writes half of the same sector)
+        even_region[odd ? 1 : 0] = pc[2 * h];
+        odd_region[odd ? 1 : 0] = pc[2 * h + 1];
       }
     }
   }
@@ -441,8 +469,13 @@ __global__ void __launch_bounds__(kQThreads) qnaive_decode_kernel(const QArgs a)
   const bool pow2 = (__float_as_uint(a.prescale) & 0x007fffffu) == 0u && (__float_as_uint(a.prescale) >> 23) - 2u < 250u;
   const float rc = pow2 ? __frcp_rn(a.prescale) : 0.0f;
   if ((b == 6u || b == 8u) && C % 1024u == 0u) {
-    if (b == 6u) qnaive_decode_rows_fast<BF16, 6>(a, lane, warp, n_warps, pow2, rc);
-    else qnaive_decode_rows_fast<BF16, 8>(a, lane, warp, n_warps, pow2, rc);
+    if (b == 6u) {
+      if (pow2) qnaive_decode_rows_fast<BF16, 6, true>(a, lane, warp, n_warps, rc);
+      else qnaive_decode_rows_fast<BF16, 6, false>(a, lane, warp, n_warps, rc);
+    } else {
+      if (pow2) qnaive_decode_rows_fast<BF16, 8, true>(a, lane, warp, n_warps, rc);
+      else qnaive_decode_rows_fast<BF16, 8, false>(a, lane, warp, n_warps, rc);
+    }
     return;
   }
   for (uint64_t r = warp; r < a.tokens; r += n_warps) {
